@@ -1,0 +1,68 @@
+// Shared host/device helpers of the cprune library (status word, error capture, bf16 vectors).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cprune.h"
+
+namespace cprune {
+
+// bits of the device status word
+enum : int { STATUS_TIMEOUT = 1, STATUS_BAD_DATA = 2 };
+
+// Device address of the per-device status word (resolved once per device).
+int *device_status_word();
+
+// Records a failing CUDA call for cprune_last_cuda_error() and returns CPRUNE_ERR_CUDA.
+cprune_status cuda_fail(cudaError_t e, const char *what);
+
+#define CPRUNE_CUDA_CHECK(expr)                                     \
+    do {                                                            \
+        cudaError_t e__ = (expr);                                   \
+        if (e__ != cudaSuccess) return ::cprune::cuda_fail(e__, #expr); \
+    } while (0)
+
+#define CPRUNE_LAUNCH_CHECK(name)                                   \
+    do {                                                            \
+        cudaError_t e__ = cudaGetLastError();                       \
+        if (e__ != cudaSuccess) return ::cprune::cuda_fail(e__, name); \
+    } while (0)
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
+
+__device__ __forceinline__ float apply_act(float v, int act) {
+    if (act == CPRUNE_ACT_RELU) return fmaxf(v, 0.f);
+    if (act == CPRUNE_ACT_RELU6) return fminf(fmaxf(v, 0.f), 6.f);
+    return v;
+}
+
+// 8 bf16 values carried in one 16-byte vector
+struct alignas(16) bf16x8 {
+    __nv_bfloat162 v[4];
+};
+
+__device__ __forceinline__ bf16x8 ldg8(const bf16x8 *p) {
+    uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
+    return *reinterpret_cast<bf16x8 *>(&u);
+}
+
+__device__ __forceinline__ void unpack8(const bf16x8 &a, float *f) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 t = __bfloat1622float2(a.v[i]);
+        f[2 * i] = t.x;
+        f[2 * i + 1] = t.y;
+    }
+}
+
+__device__ __forceinline__ bf16x8 pack8(const float *f) {
+    bf16x8 r;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r.v[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return r;
+}
+
+}  // namespace cprune

@@ -1,0 +1,488 @@
+// Dense conv task as an implicit GEMM on the sm_100a tensor cores (paper Sec. 3.4: a task is
+// Conv2d + folded BatchNorm + activation; Sec. 3.5: the filter count K is whatever pruning left).
+//
+//   D[m][k] = sum over (r, s, c) of  X[pixel m shifted by tap (r,s)][c] * Wt[k][r][s][c]
+//   m = output pixel (n, p, q) linearised,  GEMM-M = N*P*Q,  GEMM-N = K,  GEMM-K = R*S*C
+//
+// One persistent CTA per SM, 192 threads, three roles:
+//   warp 0      producer: per (tap, 64-channel block) one im2col TMA load of 128 pixels x 64
+//               channels of the activation tensor (zero fill for the padding border and for
+//               channels beyond c_pad) and one tiled TMA load of BN filters x 64 channels,
+//               both into 128-byte-swizzled shared memory, completion on an mbarrier;
+//   warp 1      issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction, bf16 x bf16 ->
+//               float32) with the accumulator in tensor memory; two accumulator buffers so
+//               that the epilogue of one tile overlaps the main loop of the next;
+//   warps 2..5  epilogue: tcgen05.ld the accumulator, add bias (+ residual), activation,
+//               convert to bf16 and store NHWC rows.
+// Odd channel counts: C is padded to a multiple of 8 in memory, the last channel block issues
+// only ceil(remaining/16) MMAs; K is covered by tiles_n tiles of BN (a multiple of 16).
+// Every wait is bounded: when a limit expires the CTA raises STATUS_TIMEOUT in the device status
+// word, all roles leave their loops, tensor memory is released and the kernel returns.
+#include <cuda.h>
+
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "plan.h"
+
+namespace cprune {
+
+constexpr int TC_THREADS = 192;
+constexpr int BM = 128;            // pixels per tile (MMA M)
+constexpr int BK = 64;             // channels per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int TMEM_COLS = 512;
+constexpr int ACC_STRIDE = 256;    // column offset of the second accumulator buffer
+constexpr int MAX_STAGES = 8;
+constexpr long long WAIT_LIMIT_CYCLES = 1LL << 31;   // about a second
+
+struct TcParams {
+    long long M;
+    int P, Q, stride, pad, R, S;
+    int cblks;         // ceil(c_pad / 64)
+    int ksteps_last;   // 16-channel MMA steps in the last channel block
+    int BN, tiles_m, tiles_n, k_pad, stages, act;
+    const float *bias;
+    const __nv_bfloat16 *res;
+    __nv_bfloat16 *y;
+    int *status;
+};
+
+// ------------------------------------------------------------------------------------------ PTX
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
+// Bounded wait.  Returns false when the limit expired here or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            atomicOr(status, STATUS_TIMEOUT);
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h,
+                                                int n, uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        :
+        : "r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        :
+        : "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :
+        : "r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t *v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, 128-byte
+// swizzled, with 8-row groups 1024 bytes apart (the layout both TMA loads produce).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);   // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                  // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                  // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                  // 128-byte swizzle
+    return d;
+}
+
+// ---------------------------------------------------------------------------------------- kernel
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
+    uint8_t *smem = smem_raw + (base - raw);
+    const int stage_bytes = A_STAGE_BYTES + p.BN * BK * 2;
+    uint8_t *ctrl = smem + (size_t)p.stages * stage_bytes;
+    const uint32_t bar0 = base + (uint32_t)p.stages * stage_bytes;
+    // barrier slots (8 bytes each): full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2]
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + 2 + a); };
+    uint32_t *tmem_slot = (uint32_t *)(ctrl + 8 * (2 * MAX_STAGES + 4));
+    volatile int *abort_flag = (volatile int *)(ctrl + 8 * (2 * MAX_STAGES + 4) + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int total_tiles = p.tiles_m * p.tiles_n;
+    const int PQ = p.P * p.Q;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
+            const long long m0 = (long long)mt * BM;
+            const int n_img = (int)(m0 / PQ);
+            const int rem = (int)(m0 - (long long)n_img * PQ);
+            const int p0 = rem / p.Q, q0 = rem - p0 * p.Q;
+            const int wc = q0 * p.stride - p.pad, hc = p0 * p.stride - p.pad;
+            for (int r = 0; r < p.R && ok; ++r)
+                for (int s = 0; s < p.S && ok; ++s)
+                    for (int cb = 0; cb < p.cblks; ++cb) {
+                        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            const uint32_t a_dst = base + (uint32_t)stage * stage_bytes;
+                            mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
+                            tma_load_im2col(a_dst, &tm_a, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
+                            tma_load_3d(a_dst + A_STAGE_BYTES, &tm_b, full_bar(stage), cb * BK, r * p.S + s, nt * p.BN);
+                        }
+                        __syncwarp();
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issue
+        // instruction descriptor: D float32, A and B bf16, both K-major, N = BN, M = 128
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_STRIDE);
+            uint32_t accumulate = 0;
+            for (int tap = 0; tap < p.R * p.S && ok; ++tap)
+                for (int cb = 0; cb < p.cblks; ++cb) {
+                    ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a_addr = base + (uint32_t)stage * stage_bytes;
+                        const uint64_t da = smem_desc_sw128(a_addr);
+                        const uint64_t db = smem_desc_sw128(a_addr + A_STAGE_BYTES);
+                        const int nk = (cb == p.cblks - 1) ? p.ksteps_last : BK / 16;
+                        for (int kk = 0; kk < nk; ++kk) {
+                            // 16 channels = 32 bytes further along the swizzled row: +2 in 16-byte units
+                            umma_bf16(d_tmem, da + (uint64_t)(2 * kk), db + (uint64_t)(2 * kk), idesc, accumulate);
+                            accumulate = 1;
+                        }
+                        umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    }
+                    __syncwarp();
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            if (ok && lane == 0) umma_commit(tfull_bar(acc));
+            __syncwarp();
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+        const int row = quarter * 32 + lane;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
+            const long long m = (long long)mt * BM + row;
+            ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * ACC_STRIDE);
+            const bool row_ok = m < p.M;
+            __nv_bfloat16 *yrow = p.y + (size_t)(row_ok ? m : 0) * p.k_pad;
+            const __nv_bfloat16 *rrow = p.res ? p.res + (size_t)(row_ok ? m : 0) * p.k_pad : nullptr;
+            for (int c0 = 0; c0 < p.BN; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(t_row + (uint32_t)c0, v);
+                tmem_ld_wait();
+                const int kg = nt * p.BN + c0;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int k0 = kg + half * 8;
+                    if (row_ok && k0 < p.k_pad) {
+                        float f[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[half * 8 + j]) + __ldg(p.bias + k0 + j);
+                        if (rrow) {
+                            float rf[8];
+                            unpack8(ldg8((const bf16x8 *)(rrow + k0)), rf);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) f[j] += rf[j];
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], p.act);
+                        *(bf16x8 *)(yrow + k0) = pack8(f);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {
+        // give copies that may still be in flight time to land before the CTA's memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn g_encode_tiled = nullptr;
+static EncodeIm2colFn g_encode_im2col = nullptr;
+static int g_driver_version = 0;
+
+static cprune_status load_driver_entry_points() {
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    if (g_encode_tiled && g_encode_im2col) return CPRUNE_OK;
+    cudaDriverEntryPointQueryResult q;
+    void *fn = nullptr;
+    CPRUNE_CUDA_CHECK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown, "cuTensorMapEncodeTiled not found");
+    g_encode_tiled = (EncodeTiledFn)fn;
+    fn = nullptr;
+    CPRUNE_CUDA_CHECK(cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorUnknown, "cuTensorMapEncodeIm2col not found");
+    g_encode_im2col = (EncodeIm2colFn)fn;
+    CPRUNE_CUDA_CHECK(cudaDriverGetVersion(&g_driver_version));
+    return CPRUNE_OK;
+}
+
+static int smem_for(int stages, int BN) {
+    return 1024 /* alignment slack */ + stages * (A_STAGE_BYTES + BN * BK * 2) + 8 * (2 * MAX_STAGES + 4) + 16;
+}
+
+// Chooses the N tile and the pipeline depth.  Eligible: dense, c_pad >= 8, im2col corner limits.
+cprune_status plan_conv_tensor(cprune_plan *plan) {
+    cprune_plan_info &i = plan->info;
+    if (i.groups != 1) return CPRUNE_ERR_UNSUPPORTED;
+    if (i.R > 16 || i.S > 16 || i.pad > 64 || i.stride > 8) return CPRUNE_ERR_UNSUPPORTED;
+    if (i.W > 65535 || i.H > 65535) return CPRUNE_ERR_UNSUPPORTED;
+    const long long M = (long long)i.N * i.P * i.Q;
+    const int tiles_m = (int)ceil_div(M, BM);
+    const int k16 = round_up(i.K, 16);
+    // fewest N tiles that fit the 256-column accumulator, then split further while that fills
+    // more of the 148 SMs without dropping below 64 columns per tile
+    int tiles_n = (k16 + 255) / 256;
+    while (true) {
+        int next = tiles_n + 1;
+        int bn_next = round_up((k16 + next - 1) / next, 16);
+        if (bn_next < 64) break;
+        if ((long long)tiles_m * tiles_n >= 148) break;
+        tiles_n = next;
+    }
+    int BN = round_up((k16 + tiles_n - 1) / tiles_n, 16);
+    tiles_n = (k16 + BN - 1) / BN;
+    int stages = MAX_STAGES;
+    while (stages > 2 && smem_for(stages, BN) > 200 * 1024) --stages;
+    i.tile_m = BM;
+    i.tile_n = BN;
+    i.tile_k = BK;
+    i.stages = stages;
+    i.tiles_m = tiles_m;
+    i.tiles_n = tiles_n;
+    i.k_alloc = tiles_n * BN;
+    const int cblks = (i.c_pad + BK - 1) / BK;
+    const int ksteps = (cblks - 1) * (BK / 16) + (i.c_pad - (cblks - 1) * BK + 15) / 16;
+    i.padded_flops = 2.0 * (double)tiles_m * BM * (double)i.k_alloc * (double)(i.R * i.S) * ksteps * 16.0;
+    plan->smem_bytes = smem_for(stages, BN);
+    return CPRUNE_OK;
+}
+
+static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w) {
+    const cprune_plan_info &i = plan->info;
+    cprune_status st = load_driver_entry_points();
+    if (st != CPRUNE_OK) return st;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)i.c_pad, (cuuint64_t)i.W, (cuuint64_t)i.H, (cuuint64_t)i.N};
+        cuuint64_t strides[3] = {(cuuint64_t)i.c_pad * 2, (cuuint64_t)i.W * i.c_pad * 2, (cuuint64_t)i.H * i.W * i.c_pad * 2};
+        int lower[2] = {-i.pad, -i.pad};
+        int upper[2] = {i.pad - (i.S - 1), i.pad - (i.R - 1)};
+        cuuint32_t estr[4] = {1, (cuuint32_t)i.stride, (cuuint32_t)i.stride, 1};
+        CUresult r = g_encode_im2col(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides,
+                                     lower, upper, BK, BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeIm2col");
+        // Drivers up to 13.1 set a descriptor bit for im2col maps of tensors smaller than 128 KiB
+        // that makes the load misbehave; the open-source CUTLASS im2col path clears it the same way.
+        const size_t bytes = (size_t)i.N * i.H * i.W * i.c_pad * 2;
+        if (g_driver_version <= 13010 && bytes < 131072) reinterpret_cast<uint64_t *>(&plan->tm_a)[1] &= ~(1ull << 21);
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)i.c_pad, (cuuint64_t)(i.R * i.S), (cuuint64_t)i.k_alloc};
+        cuuint64_t strides[2] = {(cuuint64_t)i.c_pad * 2, (cuuint64_t)i.R * i.S * i.c_pad * 2};
+        cuuint32_t box[3] = {BK, 1, (cuuint32_t)i.tile_n};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = g_encode_tiled(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box,
+                                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    }
+    plan->map_x = x;
+    plan->map_w = w;
+    return CPRUNE_OK;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    }
+    return n;
+}
+
+cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
+                                 void *y, cudaStream_t st) {
+    const cprune_plan_info &i = plan->info;
+    CUtensorMap tm_a, tm_b;
+    {
+        std::lock_guard<std::mutex> lock(plan->mu);
+        if (plan->map_x != x || plan->map_w != w) {
+            cprune_status s = encode_maps(plan, x, w);
+            if (s != CPRUNE_OK) return s;
+        }
+        std::memcpy(&tm_a, &plan->tm_a, sizeof(CUtensorMap));
+        std::memcpy(&tm_b, &plan->tm_b, sizeof(CUtensorMap));
+    }
+    static std::mutex attr_mu;
+    static int attr_set = 0;
+    {
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (!attr_set) {
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            attr_set = 1;
+        }
+    }
+    TcParams p;
+    p.M = (long long)i.N * i.P * i.Q;
+    p.P = i.P; p.Q = i.Q; p.stride = i.stride; p.pad = i.pad; p.R = i.R; p.S = i.S;
+    p.cblks = (i.c_pad + BK - 1) / BK;
+    p.ksteps_last = (i.c_pad - (p.cblks - 1) * BK + 15) / 16;
+    p.BN = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
+    p.act = plan->opts.activation;
+    p.bias = b;
+    p.res = (const __nv_bfloat16 *)res;
+    p.y = (__nv_bfloat16 *)y;
+    p.status = device_status_word();
+    if (!p.status) return cuda_fail(cudaGetLastError(), "status word");
+    const int total = i.tiles_m * i.tiles_n;
+    if (total == 0) return CPRUNE_OK;
+    const int grid = total < sm_count() ? total : sm_count();
+    conv_tc_kernel<<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_a, tm_b, p);
+    CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
+    return CPRUNE_OK;
+}
+
+}  // namespace cprune

@@ -1,0 +1,220 @@
+// Whole-model runner: the aggregate of a network's tasks enqueued back to back on one stream
+// (paper Sec. 3.1: the model is the aggregate of its tasks' programs and is timed as a whole),
+// optionally replayed as a CUDA graph so that one replay costs one host call.
+#include <map>
+#include <vector>
+
+#include "common.cuh"
+#include "plan.h"
+
+struct ModelTensor {
+    int n = 0, h = 0, w = 0, c = 0, c_pad = 0;
+    size_t offset = 0, bytes = 0;
+    bool defined = false;
+};
+
+struct cprune_model {
+    int N, H, W, C;
+    std::vector<cprune_task_desc> tasks;
+    std::map<int, ModelTensor> tensors;
+    char *arena = nullptr;
+    size_t arena_bytes = 0;
+    char *workspace = nullptr;
+    size_t workspace_bytes = 0;
+    int classes = 0;
+    int launches = 0;
+    cudaGraphExec_t exec = nullptr;
+    const float *graph_x = nullptr;
+    float *graph_logits = nullptr;
+    cudaStream_t graph_stream = nullptr;
+};
+
+namespace cprune {
+
+static size_t align256(size_t v) { return (v + 255) / 256 * 256; }
+
+static void *tensor_ptr(const cprune_model *m, int id) {
+    auto it = m->tensors.find(id);
+    return it == m->tensors.end() ? nullptr : (void *)(m->arena + it->second.offset);
+}
+
+static cprune_status enqueue(cprune_model *m, const float *x, float *logits, cudaStream_t st) {
+    cprune_status s = cprune_cast_input(x, (size_t)m->N * m->H * m->W, m->C, tensor_ptr(m, 0), st);
+    if (s != CPRUNE_OK) return s;
+    for (size_t t = 0; t < m->tasks.size(); ++t) {
+        const cprune_task_desc &d = m->tasks[t];
+        const ModelTensor &in = m->tensors[d.in];
+        void *pin = tensor_ptr(m, d.in);
+        const bool last = t + 1 == m->tasks.size();
+        void *pout = last ? (void *)logits : tensor_ptr(m, d.out);
+        switch (d.op) {
+            case CPRUNE_OP_CONV:
+                s = cprune_task_run(d.plan, pin, d.w, d.b, d.res >= 0 ? tensor_ptr(m, d.res) : nullptr, pout,
+                                    m->workspace, st);
+                break;
+            case CPRUNE_OP_MAXPOOL:
+                s = cprune_maxpool(pin, in.n, in.h, in.w, in.c, d.p0, d.p1, d.p2, pout, st);
+                break;
+            case CPRUNE_OP_GAP:
+                s = cprune_global_avgpool(pin, in.n, in.h, in.w, in.c, pout, st);
+                break;
+            case CPRUNE_OP_FC:
+                s = cprune_fc(pin, in.n, d.p0, d.w, d.b, d.p1, d.p2, last ? 1 : 0, pout, st);
+                break;
+            default:
+                s = CPRUNE_ERR_INTERNAL;
+        }
+        if (s != CPRUNE_OK) return s;
+    }
+    return CPRUNE_OK;
+}
+
+}  // namespace cprune
+
+using namespace cprune;
+
+extern "C" {
+
+cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_desc *tasks, int n_tasks,
+                                  cprune_model **out) {
+    if (!out) return CPRUNE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || !tasks || n_tasks <= 0) return CPRUNE_ERR_INVALID_ARG;
+    if (tasks[n_tasks - 1].op != CPRUNE_OP_FC) return CPRUNE_ERR_INVALID_ARG;
+    cprune_model *m = new cprune_model();
+    m->N = N; m->H = H; m->W = W; m->C = C;
+    m->tasks.assign(tasks, tasks + n_tasks);
+    ModelTensor t0;
+    t0.n = N; t0.h = H; t0.w = W; t0.c = C; t0.c_pad = cprune_padded_channels(C); t0.defined = true;
+    m->tensors[0] = t0;
+    m->launches = 1;
+    cprune_status st = CPRUNE_OK;
+    for (int t = 0; t < n_tasks && st == CPRUNE_OK; ++t) {
+        const cprune_task_desc &d = m->tasks[t];
+        auto it = m->tensors.find(d.in);
+        if (it == m->tensors.end() || d.out <= 0) { st = CPRUNE_ERR_INVALID_ARG; break; }
+        const ModelTensor in = it->second;
+        ModelTensor o;
+        o.n = in.n; o.defined = true;
+        switch (d.op) {
+            case CPRUNE_OP_CONV: {
+                if (!d.plan || !d.w || !d.b) { st = CPRUNE_ERR_INVALID_ARG; break; }
+                const cprune_plan_info &i = d.plan->info;
+                if (i.N != in.n || i.H != in.h || i.W != in.w || i.C != in.c) { st = CPRUNE_ERR_INVALID_ARG; break; }
+                if ((d.plan->opts.residual != 0) != (d.res >= 0)) { st = CPRUNE_ERR_INVALID_ARG; break; }
+                if (d.res >= 0) {
+                    auto r = m->tensors.find(d.res);
+                    if (r == m->tensors.end() || r->second.h != i.P || r->second.w != i.Q || r->second.c != i.K) {
+                        st = CPRUNE_ERR_INVALID_ARG;
+                        break;
+                    }
+                }
+                o.h = i.out_h; o.w = i.out_w; o.c = i.K;
+                if (i.workspace_bytes > m->workspace_bytes) m->workspace_bytes = i.workspace_bytes;
+                m->launches += d.plan->opts.pool ? 2 : 1;
+                break;
+            }
+            case CPRUNE_OP_MAXPOOL:
+                if (d.p0 <= 0 || d.p1 <= 0 || d.p2 < 0 || in.h + 2 * d.p2 < d.p0 || in.w + 2 * d.p2 < d.p0) {
+                    st = CPRUNE_ERR_INVALID_ARG;
+                    break;
+                }
+                o.h = (in.h + 2 * d.p2 - d.p0) / d.p1 + 1; o.w = (in.w + 2 * d.p2 - d.p0) / d.p1 + 1; o.c = in.c;
+                m->launches += 1;
+                break;
+            case CPRUNE_OP_GAP:
+                o.h = 1; o.w = 1; o.c = in.c;
+                m->launches += 1;
+                break;
+            case CPRUNE_OP_FC:
+                if (!d.w || !d.b || in.h * in.w != 1 || in.c != d.p0 || d.p1 <= 0) { st = CPRUNE_ERR_INVALID_ARG; break; }
+                o.h = 1; o.w = 1; o.c = d.p1;
+                m->launches += 1;
+                if (t == n_tasks - 1) m->classes = d.p1;
+                break;
+            default:
+                st = CPRUNE_ERR_INVALID_ARG;
+        }
+        if (st != CPRUNE_OK) break;
+        o.c_pad = cprune_padded_channels(o.c);
+        if (m->tensors.count(d.out)) { st = CPRUNE_ERR_INVALID_ARG; break; }   // single assignment
+        m->tensors[d.out] = o;
+    }
+    if (st != CPRUNE_OK) { delete m; return st; }
+    size_t off = 0;
+    for (auto &kv : m->tensors) {
+        kv.second.bytes = (size_t)kv.second.n * kv.second.h * kv.second.w * kv.second.c_pad * 2;
+        kv.second.offset = off;
+        off += align256(kv.second.bytes);
+    }
+    m->arena_bytes = off;
+    cudaError_t e = cudaMalloc((void **)&m->arena, m->arena_bytes);
+    if (e == cudaSuccess && m->workspace_bytes) e = cudaMalloc((void **)&m->workspace, m->workspace_bytes);
+    if (e != cudaSuccess) {
+        if (m->arena) cudaFree(m->arena);
+        delete m;
+        return cuda_fail(e, "cudaMalloc(model activations)");
+    }
+    *out = m;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_model_run(cprune_model *m, const float *x, float *logits, int use_graph, void *stream) {
+    if (!m || !x || !logits) return CPRUNE_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!use_graph) return enqueue(m, x, logits, st);
+    if (m->exec && m->graph_x == x && m->graph_logits == logits && m->graph_stream == st) {
+        CPRUNE_CUDA_CHECK(cudaGraphLaunch(m->exec, st));
+        return CPRUNE_OK;
+    }
+    if (m->exec) { cudaGraphExecDestroy(m->exec); m->exec = nullptr; }
+    // first call for this (x, logits, stream): run eagerly (this also encodes tensor maps and sets
+    // kernel attributes outside of any capture), then record the same sequence for later replays
+    cprune_status s = enqueue(m, x, logits, st);
+    if (s != CPRUNE_OK) return s;
+    cudaGraph_t graph = nullptr;
+    CPRUNE_CUDA_CHECK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    s = enqueue(m, x, logits, st);
+    cudaError_t e = cudaStreamEndCapture(st, &graph);
+    if (s != CPRUNE_OK) { if (graph) cudaGraphDestroy(graph); return s; }
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
+    e = cudaGraphInstantiate(&m->exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { m->exec = nullptr; return cuda_fail(e, "cudaGraphInstantiate"); }
+    m->graph_x = x; m->graph_logits = logits; m->graph_stream = st;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_model_tensor(const cprune_model *m, int id, const void **ptr, int *n, int *h, int *w, int *c_pad) {
+    if (!m) return CPRUNE_ERR_INVALID_ARG;
+    auto it = m->tensors.find(id);
+    if (it == m->tensors.end()) return CPRUNE_ERR_INVALID_ARG;
+    if (ptr) *ptr = m->arena + it->second.offset;
+    if (n) *n = it->second.n;
+    if (h) *h = it->second.h;
+    if (w) *w = it->second.w;
+    if (c_pad) *c_pad = it->second.c_pad;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_model_copy_tensor(const cprune_model *m, int id, void *dst, void *stream) {
+    if (!m || !dst) return CPRUNE_ERR_INVALID_ARG;
+    auto it = m->tensors.find(id);
+    if (it == m->tensors.end()) return CPRUNE_ERR_INVALID_ARG;
+    CPRUNE_CUDA_CHECK(cudaMemcpyAsync(dst, m->arena + it->second.offset, it->second.bytes, cudaMemcpyDeviceToDevice,
+                                      (cudaStream_t)stream));
+    return CPRUNE_OK;
+}
+
+int cprune_model_launches(const cprune_model *m) { return m ? m->launches : 0; }
+
+cprune_status cprune_model_destroy(cprune_model *m) {
+    if (!m) return CPRUNE_ERR_INVALID_ARG;
+    if (m->exec) cudaGraphExecDestroy(m->exec);
+    if (m->arena) cudaFree(m->arena);
+    if (m->workspace) cudaFree(m->workspace);
+    delete m;
+    return CPRUNE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,185 @@
+// Task plans and the plan cache (paper Sec. 3.1 / Sec. 3.4: subgraphs with identical shape and
+// properties map to one task, and each task keeps one program).  A plan is a pure function of its
+// key (shape + fused-epilogue options); planning launches nothing and needs no device.
+#include <array>
+#include <map>
+#include <mutex>
+
+#include "common.cuh"
+#include "plan.h"
+
+namespace cprune {
+
+using PlanKey = std::array<int, 14>;
+
+struct PlanCache {
+    std::mutex mu;
+    std::map<PlanKey, cprune_plan *> plans;
+    long long hits = 0;
+};
+
+static PlanCache &cache() {
+    static PlanCache c;
+    return c;
+}
+
+static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
+    cprune_plan *pl = new cprune_plan();
+    cprune_plan_info &i = pl->info;
+    i = cprune_plan_info();
+    i.N = key[0]; i.C = key[1]; i.H = key[2]; i.W = key[3]; i.K = key[4]; i.R = key[5]; i.S = key[6];
+    i.stride = key[7]; i.pad = key[8]; i.groups = key[9];
+    pl->opts.activation = key[10]; pl->opts.residual = key[11]; pl->opts.pool = key[12]; pl->opts.kernel = key[13];
+    pl->refs = 0;
+    i.P = (i.H + 2 * i.pad - i.R) / i.stride + 1;
+    i.Q = (i.W + 2 * i.pad - i.S) / i.stride + 1;
+    i.out_h = i.P; i.out_w = i.Q;
+    if (pl->opts.pool == CPRUNE_POOL_MAX2X2) { i.out_h = i.P / 2; i.out_w = i.Q / 2; }
+    i.c_pad = cprune_padded_channels(i.C);
+    i.k_pad = cprune_padded_channels(i.K);
+    i.k_alloc = i.k_pad;
+    i.flops = 2.0 * i.N * (double)i.K * (i.C / i.groups) * i.P * i.Q * i.R * i.S;
+    i.padded_flops = 2.0 * i.N * (double)i.k_pad * (i.groups == 1 ? i.c_pad : 1) * i.P * i.Q * i.R * i.S;
+    const bool depthwise = i.groups > 1;
+    int family = pl->opts.kernel;
+    cprune_status st = CPRUNE_OK;
+    if (depthwise) {
+        if (family != CPRUNE_KERNEL_AUTO && family != CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;
+        family = CPRUNE_KERNEL_DEPTHWISE;
+        i.tile_m = 1;
+        i.tile_n = i.stride == 1 ? (i.Q >= 4 ? 4 : (i.Q >= 2 ? 2 : 1)) : (i.Q >= 2 ? 2 : 1);  // output columns per thread
+        i.tile_k = 8;
+    } else {
+        if (family == CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;
+        if (family == CPRUNE_KERNEL_AUTO) family = i.C < 8 ? CPRUNE_KERNEL_DIRECT : CPRUNE_KERNEL_TENSOR;
+        if (st == CPRUNE_OK && family == CPRUNE_KERNEL_TENSOR) {
+            cprune_status t = plan_conv_tensor(pl);
+            if (t != CPRUNE_OK) {
+                if (pl->opts.kernel == CPRUNE_KERNEL_TENSOR) st = t;
+                family = CPRUNE_KERNEL_DIRECT;
+            }
+        }
+        if (family == CPRUNE_KERNEL_DIRECT) {
+            i.tile_m = 1; i.tile_n = 8; i.tile_k = 8; i.stages = 0;
+            i.tiles_m = i.N * i.P * i.Q; i.tiles_n = i.k_pad / 8;
+        }
+    }
+    if (st != CPRUNE_OK) { delete pl; return st; }
+    i.kernel = family;
+    const double rs = (double)i.R * i.S;
+    i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * i.S * i.c_pad * 2;
+    i.packed_bias_bytes = (size_t)i.k_alloc * sizeof(float);
+    i.workspace_bytes = pl->opts.pool == CPRUNE_POOL_MAX2X2 ? (size_t)i.N * i.P * i.Q * i.k_pad * 2 : 0;
+    i.algorithmic_bytes = 2.0 * ((double)i.N * i.H * i.W * i.C + (double)i.N * i.out_h * i.out_w * i.K +
+                                 (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
+                                 (double)i.K * (i.C / i.groups) * rs) + 4.0 * i.K;
+    *out = pl;
+    return CPRUNE_OK;
+}
+
+}  // namespace cprune
+
+using namespace cprune;
+
+extern "C" {
+
+cprune_status cprune_task_plan(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int groups,
+                               const cprune_task_opts *opts, cprune_plan **out) {
+    if (!out) return CPRUNE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0 || groups <= 0)
+        return CPRUNE_ERR_INVALID_ARG;
+    if (H + 2 * pad < R || W + 2 * pad < S) return CPRUNE_ERR_INVALID_ARG;
+    cprune_task_opts o = {CPRUNE_ACT_RELU, 0, CPRUNE_POOL_NONE, CPRUNE_KERNEL_AUTO};
+    if (opts) o = *opts;
+    if (o.activation < 0 || o.activation > 2 || o.pool < 0 || o.pool > 1 || o.kernel < 0 || o.kernel > 3 ||
+        (o.residual != 0 && o.residual != 1))
+        return CPRUNE_ERR_INVALID_ARG;
+    if (groups != 1) {
+        if (groups != C || K != C) return CPRUNE_ERR_UNSUPPORTED;
+        if (R != 3 || S != 3 || stride > 2) return CPRUNE_ERR_UNSUPPORTED;
+    }
+    int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
+    if (o.pool == CPRUNE_POOL_MAX2X2 && ((P & 1) || (Q & 1))) return CPRUNE_ERR_INVALID_ARG;
+    if ((long long)N * P * Q > 0x7fffffffLL || (long long)N * H * W > 0x7fffffffLL) return CPRUNE_ERR_UNSUPPORTED;
+    PlanKey key = {N, C, H, W, K, R, S, stride, pad, groups, o.activation, o.residual, o.pool, o.kernel};
+    PlanCache &c = cache();
+    std::lock_guard<std::mutex> lock(c.mu);
+    auto it = c.plans.find(key);
+    if (it != c.plans.end()) {
+        ++c.hits;
+        ++it->second->refs;
+        *out = it->second;
+        return CPRUNE_OK;
+    }
+    cprune_plan *pl = nullptr;
+    cprune_status st = build_plan(key, &pl);
+    if (st != CPRUNE_OK) return st;
+    pl->refs = 1;
+    c.plans[key] = pl;
+    *out = pl;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_plan_query(const cprune_plan *plan, cprune_plan_info *out) {
+    if (!plan || !out) return CPRUNE_ERR_INVALID_ARG;
+    *out = plan->info;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_plan_release(cprune_plan *plan) {
+    if (!plan) return CPRUNE_ERR_INVALID_ARG;
+    PlanCache &c = cache();
+    std::lock_guard<std::mutex> lock(c.mu);
+    if (plan->refs <= 0) return CPRUNE_ERR_INVALID_ARG;
+    --plan->refs;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_cache_clear(int *n_left) {
+    PlanCache &c = cache();
+    std::lock_guard<std::mutex> lock(c.mu);
+    for (auto it = c.plans.begin(); it != c.plans.end();) {
+        if (it->second->refs == 0) {
+            delete it->second;
+            it = c.plans.erase(it);
+        } else {
+            ++it;
+        }
+    }
+    if (n_left) *n_left = (int)c.plans.size();
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_cache_stats(int *n_plans, long long *n_hits) {
+    PlanCache &c = cache();
+    std::lock_guard<std::mutex> lock(c.mu);
+    if (n_plans) *n_plans = (int)c.plans.size();
+    if (n_hits) *n_hits = c.hits;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_task_run(cprune_plan *plan, const void *x, const void *w_packed, const float *b_packed,
+                              const void *residual, void *y, void *workspace, void *stream) {
+    if (!plan || !x || !w_packed || !b_packed || !y) return CPRUNE_ERR_INVALID_ARG;
+    if ((plan->opts.residual != 0) != (residual != nullptr)) return CPRUNE_ERR_INVALID_ARG;
+    if (((uintptr_t)x | (uintptr_t)w_packed | (uintptr_t)y | (uintptr_t)residual | (uintptr_t)workspace) & 15)
+        return CPRUNE_ERR_INVALID_ARG;
+    const cprune_plan_info &i = plan->info;
+    const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
+    if (pool && !workspace) return CPRUNE_ERR_INVALID_ARG;
+    void *conv_out = pool ? workspace : y;
+    cudaStream_t st = (cudaStream_t)stream;
+    cprune_status s;
+    switch (i.kernel) {
+        case CPRUNE_KERNEL_TENSOR: s = launch_conv_tensor(plan, x, w_packed, b_packed, residual, conv_out, st); break;
+        case CPRUNE_KERNEL_DIRECT: s = launch_conv_direct(plan, x, w_packed, b_packed, residual, conv_out, st); break;
+        case CPRUNE_KERNEL_DEPTHWISE: s = launch_depthwise(plan, x, w_packed, b_packed, residual, conv_out, st); break;
+        default: return CPRUNE_ERR_INTERNAL;
+    }
+    if (s != CPRUNE_OK) return s;
+    if (pool) return launch_maxpool(conv_out, i.N, i.P, i.Q, i.k_pad, 2, 2, 0, y, st);
+    return CPRUNE_OK;
+}
+
+}  // extern "C"

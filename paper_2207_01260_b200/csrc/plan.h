@@ -1,0 +1,43 @@
+// Internal definition of a task plan and the launchers of the kernel families.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "cprune.h"
+
+struct cprune_plan {
+    cprune_plan_info info;
+    cprune_task_opts opts;
+    int refs;
+    // tensor-core family: tensor maps are encoded for a given (x, w) pointer pair and reused
+    // while the pointers stay the same
+    std::mutex mu;
+    const void *map_x = nullptr;
+    const void *map_w = nullptr;
+    alignas(64) CUtensorMap tm_a;
+    alignas(64) CUtensorMap tm_b;
+    int smem_bytes = 0;
+};
+
+namespace cprune {
+
+// CUDA-core direct convolution, any dense shape (fallback family and small-C stems)
+cprune_status launch_conv_direct(const cprune_plan *plan, const void *x, const void *w, const float *b,
+                                 const void *res, void *y, cudaStream_t st);
+// depthwise 3x3
+cprune_status launch_depthwise(const cprune_plan *plan, const void *x, const void *w, const float *b,
+                               const void *res, void *y, cudaStream_t st);
+// tcgen05 implicit GEMM
+cprune_status plan_conv_tensor(cprune_plan *plan);  // fills tile fields of plan->info; UNSUPPORTED if not eligible
+cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
+                                 void *y, cudaStream_t st);
+// 2x2 stride-2 max-pool as a separate pass (used when a plan asks for a pool and the conv kernel
+// does not fuse it): x [N][H][W][c] -> y [N][H/2][W/2][c]
+cprune_status launch_maxpool(const void *x, int N, int H, int W, int c_pad, int k, int stride, int pad, void *y,
+                             cudaStream_t st);
+
+}  // namespace cprune

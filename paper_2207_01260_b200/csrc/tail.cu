@@ -1,0 +1,149 @@
+// Model-tail operators on bf16 NHWC tensors with padded channels: k x k max-pool, global
+// average pool and fully-connected layers.  All are memory-bound; float32 arithmetic.
+#include "common.cuh"
+#include "plan.h"
+
+namespace cprune {
+
+__global__ void __launch_bounds__(256) maxpool_kernel(const bf16x8 *__restrict__ x, int N, int H, int W, int c8,
+                                                      int P, int Q, int k, int stride, int pad,
+                                                      bf16x8 *__restrict__ y) {
+    long long total = (long long)N * P * Q * c8;
+    long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    int cg = (int)(e % c8);
+    long long t = e / c8;
+    int q = (int)(t % Q);
+    t /= Q;
+    int p = (int)(t % P);
+    int n = (int)(t / P);
+    float m[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m[i] = -INFINITY;
+    for (int r = 0; r < k; ++r) {
+        int h = p * stride - pad + r;
+        if (h < 0 || h >= H) continue;
+        for (int s = 0; s < k; ++s) {
+            int v = q * stride - pad + s;
+            if (v < 0 || v >= W) continue;
+            float f[8];
+            unpack8(ldg8(x + (((size_t)n * H + h) * W + v) * c8 + cg), f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], f[i]);
+        }
+    }
+    y[e] = pack8(m);
+}
+
+// one thread per (n, channel group): mean over H*W in float32, stored as bf16
+__global__ void __launch_bounds__(128) gap_kernel(const bf16x8 *__restrict__ x, int N, int HW, int c8,
+                                                  bf16x8 *__restrict__ y) {
+    int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= N * c8) return;
+    int cg = e % c8, n = e / c8;
+    float s[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = 0.f;
+    const bf16x8 *px = x + (size_t)n * HW * c8 + cg;
+    for (int i = 0; i < HW; ++i) {
+        float f[8];
+        unpack8(ldg8(px + (size_t)i * c8), f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j] += f[j];
+    }
+    float inv = 1.f / (float)HW;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s[j] *= inv;
+    y[e] = pack8(s);
+}
+
+// one warp per output feature o, looping over the images of the batch in groups of NB so that a
+// weight row is read once per group
+template <int NB>
+__global__ void __launch_bounds__(256) fc_kernel(const bf16x8 *__restrict__ x, int N, int in8,
+                                                 const bf16x8 *__restrict__ w, const float *__restrict__ b, int out,
+                                                 int out_pad, int act, int out_is_f32, void *__restrict__ y) {
+    int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    int lane = threadIdx.x & 31;
+    if (o >= out_pad) return;
+    const bf16x8 *wr = w + (size_t)o * in8;
+    for (int n0 = 0; n0 < N; n0 += NB) {
+        float acc[NB];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) acc[j] = 0.f;
+        for (int i = lane; i < in8; i += 32) {
+            float wf[8];
+            unpack8(ldg8(wr + i), wf);
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                if (n0 + j < N) {
+                    float xf[8];
+                    unpack8(ldg8(x + (size_t)(n0 + j) * in8 + i), xf);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) acc[j] = fmaf(xf[t], wf[t], acc[j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            float v = acc[j];
+            for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+            if (lane == 0 && n0 + j < N) {
+                v = apply_act(v + b[o], act);
+                if (out_is_f32) {
+                    if (o < out) ((float *)y)[(size_t)(n0 + j) * out + o] = v;
+                } else {
+                    ((__nv_bfloat16 *)y)[(size_t)(n0 + j) * out_pad + o] = __float2bfloat16_rn(o < out ? v : 0.f);
+                }
+            }
+        }
+    }
+}
+
+cprune_status launch_maxpool(const void *x, int N, int H, int W, int c_pad, int k, int stride, int pad, void *y,
+                             cudaStream_t st) {
+    int P = (H + 2 * pad - k) / stride + 1, Q = (W + 2 * pad - k) / stride + 1;
+    long long total = (long long)N * P * Q * (c_pad / 8);
+    if (total == 0) return CPRUNE_OK;
+    long long blocks = ceil_div(total, 256);
+    if (blocks > 0x7fffffffLL) return CPRUNE_ERR_UNSUPPORTED;
+    maxpool_kernel<<<(unsigned)blocks, 256, 0, st>>>((const bf16x8 *)x, N, H, W, c_pad / 8, P, Q, k, stride, pad,
+                                                     (bf16x8 *)y);
+    CPRUNE_LAUNCH_CHECK("maxpool_kernel");
+    return CPRUNE_OK;
+}
+
+}  // namespace cprune
+
+using namespace cprune;
+
+extern "C" {
+
+cprune_status cprune_maxpool(const void *x, int N, int H, int W, int C, int k, int stride, int pad, void *y,
+                             void *stream) {
+    if (!x || !y || N <= 0 || H <= 0 || W <= 0 || C <= 0 || k <= 0 || stride <= 0 || pad < 0 || 2 * pad > k)
+        return CPRUNE_ERR_INVALID_ARG;
+    if (H + 2 * pad < k || W + 2 * pad < k) return CPRUNE_ERR_INVALID_ARG;
+    return launch_maxpool(x, N, H, W, cprune_padded_channels(C), k, stride, pad, y, (cudaStream_t)stream);
+}
+
+cprune_status cprune_global_avgpool(const void *x, int N, int H, int W, int C, void *y, void *stream) {
+    if (!x || !y || N <= 0 || H <= 0 || W <= 0 || C <= 0) return CPRUNE_ERR_INVALID_ARG;
+    int c8 = cprune_padded_channels(C) / 8;
+    gap_kernel<<<(N * c8 + 127) / 128, 128, 0, (cudaStream_t)stream>>>((const bf16x8 *)x, N, H * W, c8, (bf16x8 *)y);
+    CPRUNE_LAUNCH_CHECK("gap_kernel");
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_fc(const void *x, int N, int in, const void *w_packed, const float *b_packed, int out, int act,
+                        int out_is_f32, void *y, void *stream) {
+    if (!x || !w_packed || !b_packed || !y || N <= 0 || in <= 0 || out <= 0) return CPRUNE_ERR_INVALID_ARG;
+    int in8 = cprune_padded_channels(in) / 8, out_pad = cprune_padded_channels(out);
+    int warps = 8;
+    fc_kernel<8><<<(out_pad + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(
+        (const bf16x8 *)x, N, in8, (const bf16x8 *)w_packed, b_packed, out, out_pad, act, out_is_f32, y);
+    CPRUNE_LAUNCH_CHECK("fc_kernel");
+    return CPRUNE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,143 @@
+"""Builds and runs a whole pruned network through the C ABI.
+
+Given a layer table (see ``workloads``) and the full-width float32 parameters, this module
+  1. uploads the parameters,
+  2. prunes every layer that has a keep count with ``cprune_select_filters`` and slices all of its
+     consumers with the gather calls (paper Sec. 3.5: L1-norm ranking, then the next layer's input
+     channels follow),
+  3. plans and packs every conv task, packs the FC layers,
+  4. assembles the task list and creates a ``cprune_model``.
+It only sequences library calls and keeps device buffers alive; all arithmetic runs in the kernels.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class PrunedNetwork:
+    def __init__(self, table: dict, weights: dict, batch: int, device="cuda:0", kernel="auto"):
+        self.table, self.batch, self.device = table, batch, torch.device(device)
+        self.kernel = kernel
+        self.params = {k: (torch.from_numpy(np.ascontiguousarray(w)).to(self.device),
+                           torch.from_numpy(np.ascontiguousarray(b)).to(self.device)) for k, (w, b) in weights.items()}
+        self.kept = {}
+        self._by = {l["name"]: l for l in table["layers"]}
+        self._prune()
+        self._assemble()
+
+    # ---------------------------------------------------------------- pruning
+    def _follow(self, layer, kept, first_done):
+        """Slice the consumers of `layer` by `kept`; the first consumer was already handled by
+        cprune_select_filters itself when first_done is set."""
+        for i, (cname, how) in enumerate(layer["consumers"]):
+            w, b = self.params[cname]
+            if how in ("in_channels", "fc_in"):
+                if not (first_done and i == 0):
+                    self.params[cname] = (B.cprune_gather_columns(w, kept), b)
+            elif how == "depthwise":
+                if not (first_done and i == 0):
+                    w = B.cprune_gather_rows(w, kept)
+                    self.params[cname] = (w, b)
+                self.params[cname] = (self.params[cname][0], B.cprune_gather_rows(b, kept))
+                self._follow(self._by[cname], kept, False)
+            else:
+                raise ValueError(how)
+
+    def _prune(self):
+        for l in self.table["layers"]:
+            if l["kind"] != "conv" or l["keep"] is None:
+                continue
+            w, b = self.params[l["name"]]
+            w_next, dw = None, False
+            if l["consumers"]:
+                cname, how = l["consumers"][0]
+                w_next = self.params[cname][0]
+                dw = how == "depthwise"
+                if how == "fc_in":
+                    w_next = w_next.reshape(w_next.shape[0], w_next.shape[1], 1, 1)
+            kept, w_out, b_out, wn_out = B.cprune_select_filters(w, l["keep"], b, w_next, dw)
+            self.params[l["name"]] = (w_out, b_out)
+            self.kept[l["name"]] = kept
+            if l["consumers"]:
+                cname, how = l["consumers"][0]
+                if how == "fc_in":
+                    wn_out = wn_out.reshape(wn_out.shape[0], wn_out.shape[1])
+                self.params[cname] = (wn_out, self.params[cname][1])
+            self._follow(l, kept, True)
+
+    # ---------------------------------------------------------------- assembly
+    def _assemble(self):
+        H, W, C = self.table["input"]
+        ids = {"x": 0}
+        shape = {"x": (H, W, C)}
+        self.plans, self.packed, tasks = {}, {}, []
+
+        def tid(name):
+            if name not in ids:
+                ids[name] = len(ids)
+            return ids[name]
+
+        for l in self.table["layers"]:
+            kind = l["kind"]
+            h, w, c = shape[l["in"]]
+            if kind == "flatten":
+                ids[l["out"]] = ids[l["in"]]
+                shape[l["out"]] = shape[l["in"]]
+                continue
+            d = B.TaskDesc()
+            d.in_, d.out, d.res = tid(l["in"]), tid(l["out"]), -1
+            if kind == "conv":
+                wt, bs = self.params[l["name"]]
+                K, cg = wt.shape[0], wt.shape[1]
+                groups = K if l["groups"] > 1 else 1
+                assert cg * groups == c, (l["name"], cg, groups, c)
+                plan = B.cprune_task_plan(self.batch, c, h, w, K, l["R"], l["S"], l["stride"], l["pad"], groups,
+                                          l["act"], l.get("res") is not None, l.get("pool"),
+                                          self.kernel if groups == 1 else "auto")
+                wp, bp = B.cprune_pack_weights(plan, wt, bs)
+                self.plans[l["name"]], self.packed[l["name"]] = plan, (wp, bp)
+                d.op, d.plan, d.w, d.b = B.OP_CONV, plan.handle, wp.data_ptr(), bp.data_ptr()
+                if l.get("res") is not None:
+                    d.res = tid(l["res"])
+                shape[l["out"]] = (plan.out_h, plan.out_w, K)
+            elif kind == "maxpool":
+                d.op, d.p0, d.p1, d.p2 = B.OP_MAXPOOL, l["k"], l["stride"], l["pad"]
+                shape[l["out"]] = ((h + 2 * l["pad"] - l["k"]) // l["stride"] + 1,
+                                   (w + 2 * l["pad"] - l["k"]) // l["stride"] + 1, c)
+            elif kind == "gap":
+                d.op = B.OP_GAP
+                shape[l["out"]] = (1, 1, c)
+            elif kind == "fc":
+                wt, bs = self.params[l["name"]]
+                wp, bp = B.cprune_fc_pack(wt, bs)
+                self.packed[l["name"]] = (wp, bp)
+                d.op, d.w, d.b = B.OP_FC, wp.data_ptr(), bp.data_ptr()
+                d.p0, d.p1, d.p2 = wt.shape[1], wt.shape[0], B.ACT[l["act"]]
+                shape[l["out"]] = (1, 1, wt.shape[0])
+            else:
+                raise ValueError(kind)
+            tasks.append(d)
+        self.tensor_ids, self.shapes = ids, shape
+        self.model = B.cprune_model_create(self.batch, H, W, C, tasks, keep_alive=(self.plans, self.packed))
+        torch.cuda.synchronize(self.device)
+
+    # ---------------------------------------------------------------- running
+    def run(self, x, logits=None, use_graph=False):
+        """x: float32 [batch, H, W, C] device tensor -> float32 logits [batch, classes]."""
+        return B.cprune_model_run(self.model, x, logits, use_graph)
+
+    def activation(self, name):
+        """Copy of a stored activation as float32 numpy [N, h, w, c] without the pad lanes."""
+        c = self.shapes[name][2]
+        buf = self.model.copy_tensor(self.tensor_ids[name])
+        torch.cuda.synchronize(self.device)
+        return buf.float().cpu().numpy()[..., :c]
+
+    def flops(self):
+        return sum(p.flops for p in self.plans.values())
+
+    def conv_launch_info(self):
+        return {k: p.info for k, p in self.plans.items()}

@@ -1,0 +1,98 @@
+"""CPU-only checks of the library boundary: it loads, exports what the header declares, and its
+host-side logic (argument validation, plans, plan cache) behaves without a device."""
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def cp():
+    from paper_2207_01260_b200 import build
+    build.build()
+    import paper_2207_01260_b200 as m
+    m.lib()
+    return m
+
+
+def test_library_exports_every_declared_symbol(cp):
+    header = open(os.path.join(ROOT, "include", "cprune.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(cprune_[a-z0-9_]+)\s*\(", header))
+    assert len(declared) >= 25
+    assert declared == set(cp.EXPORTS)
+    L = cp.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_status_strings_and_padding(cp):
+    L = cp.lib()
+    assert L.cprune_status_string(0) == b"ok"
+    assert len({L.cprune_status_string(i) for i in range(8)}) == 8
+    assert [cp.cprune_padded_channels(c) for c in (1, 3, 8, 9, 44, 45, 243, 358)] == [8, 8, 8, 16, 48, 48, 248, 360]
+    assert cp.cprune_select_workspace_bytes(0) == 0 and cp.cprune_select_workspace_bytes(1280) >= 1280 * 12
+
+
+def test_plan_shapes_and_families(cp):
+    p = cp.cprune_task_plan(64, 64, 56, 56, 44, 3, 3, 1, 1)
+    assert (p.P, p.Q, p.c_pad, p.k_pad) == (56, 56, 64, 48)
+    assert cp.KERNEL_NAMES[p.kernel] == "tensor" and p.tile_m == 128 and p.tile_n % 16 == 0
+    assert p.tiles_m == 64 * 56 * 56 // 128 and p.tiles_n * p.tile_n >= 44 and p.k_alloc == p.tiles_n * p.tile_n
+    assert p.flops == 2.0 * 64 * 44 * 64 * 56 * 56 * 9
+    assert p.padded_flops >= p.flops
+    p = cp.cprune_task_plan(1, 3, 224, 224, 64, 7, 7, 2, 3)
+    assert (p.P, p.Q) == (112, 112) and cp.KERNEL_NAMES[p.kernel] == "direct"
+    p = cp.cprune_task_plan(8, 108, 56, 56, 108, 3, 3, 2, 1, groups=108, activation="relu6")
+    assert cp.KERNEL_NAMES[p.kernel] == "depthwise" and (p.P, p.Q) == (28, 28) and p.c_pad == 112
+    assert p.flops == 2.0 * 8 * 108 * 28 * 28 * 9
+    p = cp.cprune_task_plan(128, 45, 32, 32, 58, 3, 3, 1, 1, pool="max2x2")
+    assert (p.out_h, p.out_w) == (16, 16) and p.workspace_bytes == 128 * 32 * 32 * 64 * 2
+    # every pruned filter count gets a legal tile: N tile a multiple of 16 within the accumulator
+    for K in range(64, 513, 7):
+        p = cp.cprune_task_plan(64, 256, 14, 14, K, 3, 3, 1, 1)
+        assert p.tile_n % 16 == 0 and 16 <= p.tile_n <= 256 and p.k_alloc >= p.k_pad >= K
+        assert 2 <= p.stages <= 8
+
+
+def test_plan_cache(cp):
+    cp.cprune_cache_clear()
+    n0, h0 = cp.cprune_cache_stats()
+    a = cp.cprune_task_plan(2, 89, 28, 28, 128, 3, 3, 1, 1)
+    b = cp.cprune_task_plan(2, 89, 28, 28, 128, 3, 3, 1, 1)
+    c = cp.cprune_task_plan(2, 89, 28, 28, 128, 3, 3, 1, 1, activation="none")
+    assert a.handle.value == b.handle.value != c.handle.value
+    n1, h1 = cp.cprune_cache_stats()
+    assert n1 - n0 == 2 and h1 - h0 == 1
+    ha = a.handle.value
+    del a, b, c
+    import gc
+    gc.collect()
+    cp.cprune_cache_clear()
+    assert cp.cprune_cache_stats()[0] == n0
+    d = cp.cprune_task_plan(2, 89, 28, 28, 128, 3, 3, 1, 1)
+    assert d.info["tile_n"] > 0 and ha is not None
+
+
+def test_plan_argument_errors(cp):
+    for args in [(0, 8, 8, 8, 8, 3, 3, 1, 1), (1, 8, 8, 8, 0, 3, 3, 1, 1), (1, 8, 2, 2, 8, 7, 7, 1, 0),
+                 (1, 8, 8, 8, 8, 3, 3, 0, 1)]:
+        with pytest.raises(cp.CpruneError) as e:
+            cp.cprune_task_plan(*args)
+        assert e.value.status == 1
+    with pytest.raises(cp.CpruneError) as e:
+        cp.cprune_task_plan(1, 8, 8, 8, 8, 5, 5, 1, 2, groups=8)      # depthwise is 3x3 only
+    assert e.value.status == 2
+    with pytest.raises(cp.CpruneError) as e:
+        cp.cprune_task_plan(1, 8, 7, 7, 8, 3, 3, 1, 1, pool="max2x2")  # odd extent cannot be pooled 2x2
+    assert e.value.status == 1
+
+
+def test_missing_library_fails_loudly(cp, monkeypatch):
+    from paper_2207_01260_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libcprune.so")
+    with pytest.raises(RuntimeError):
+        binding.lib()
