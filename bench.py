@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the pruned-CNN task path on B200.
+
+A step is one pass of a whole pruned network over one batch of synthetic images: the input
+cast, every conv task (fused bias / activation / residual / pool), the pools, the global average
+pool and the FC tail -- everything `cprune_model_run` enqueues.  The one-time part of the path
+(L1 selection, slicing, weight packing) is timed separately and reported as `prepare_ms`.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet18|mobilenet_v2|vgg16_cifar]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores, same metric
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an independent replica on
+its own GPU with its own batch: weak scaling, no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOADS = {"resnet18": ("resnet18", 64), "mobilenet_v2": ("mobilenet_v2", 64), "vgg16_cifar": ("vgg16_cifar", 128)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_reference(args, table_name, batch):
+    """The oracle, as it stands, on the host cores: each step runs the pruned network on a bounded
+    sample of the batch."""
+    import oracle
+    import workloads as wl
+    table = wl.MODELS[table_name]()
+    weights = wl.model_weights(table)
+    pw, _ = oracle.prune_model(table, weights)
+    sample = {"resnet18": 2, "mobilenet_v2": 4, "vgg16_cifar": 8}[table_name]
+    sample = min(sample, batch)
+    x = wl.model_input(table, sample)
+    for _ in range(min(args.warmup, 1)):
+        oracle.model_ref(table, pw, x, matched=True)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.model_ref(table, pw, x, matched=True)
+    dt = time.perf_counter() - t0
+    return sample * args.steps / dt, dt * 1e3 / args.steps, sample, oracle.num_threads()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every launch from the host instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    table_name, batch = WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = {"workload": "pruned_%s_batch%d" % (table_name, batch), "batch_per_gpu": batch, "layout": "NHWC bf16",
+           "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
+           "l2": "activations of one step exceed the 126 MB L2 (inputs larger than L2)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, min(args.steps, 5))
+        args.steps = steps
+        v, ms, sample, cores = cpu_reference(args, table_name, batch)
+        line = {"impl": "reference", "metric": "pruned_model_images_per_s", "value": v, "unit": "images/s",
+                "n_gpus": 0, "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+                "cpu_baseline": {"value": v, "unit": "images/s", "cores": cores, "kind": "oracle",
+                                 "sample": "%d images of the %s batch per step" % (sample, cfg["workload"])},
+                "e2e": {"value": v, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2207_01260_b200 as cp
+    import workloads as wl
+    from paper_2207_01260_b200.pipeline import PrunedNetwork
+
+    cp.lib()  # fails loudly if the CUDA library is missing: there is no other path
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    table = wl.MODELS[table_name]()
+    weights = wl.model_weights(table)
+    x_host = torch.from_numpy(wl.model_input(table, batch, seed=table["seed"] + 17 * rank)).pin_memory()
+
+    t0 = time.perf_counter()
+    net = PrunedNetwork(table, weights, batch, device=dev)
+    torch.cuda.synchronize(dev)
+    prepare_first_ms = (time.perf_counter() - t0) * 1e3
+    t0 = time.perf_counter()
+    net2 = PrunedNetwork(table, weights, batch, device=dev)   # second pass: allocator and plan cache warm
+    torch.cuda.synchronize(dev)
+    prepare_ms = (time.perf_counter() - t0) * 1e3
+    del net2
+    cp.cprune_poll_device_status()
+
+    x = x_host.to(dev)
+    logits = torch.empty((batch, net.model.classes), dtype=torch.float32, device=dev)
+    logits_host = torch.empty((batch, net.model.classes), dtype=torch.float32).pin_memory()
+    use_graph = not args.no_graph
+    stream = torch.cuda.current_stream()
+
+    # ---------------- device-resident throughput
+    for _ in range(max(args.warmup, 3)):
+        net.run(x, logits, use_graph)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        net.run(x, logits, use_graph)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    cp.cprune_poll_device_status()
+
+    # ---------------- end to end: pinned host input -> device -> model -> logits back on the host
+    for _ in range(3):
+        x.copy_(x_host, non_blocking=True)
+        net.run(x, logits, use_graph)
+        logits_host.copy_(logits, non_blocking=True)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    for _ in range(args.steps):
+        x.copy_(x_host, non_blocking=True)
+        net.run(x, logits, use_graph)
+        logits_host.copy_(logits, non_blocking=True)
+    e3.record(stream)
+    barrier()
+    ms_e2e = e2.elapsed_time(e3)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+
+    # ---------------- per-task timing of the tensor-core kernel (roofline of the dominant kernel)
+    roof, per_task = None, []
+    if rank == 0:
+        peaks = measured_peaks()
+        per_task = net_task_times(cp, net, table, x, reps=5)
+        tens = [t for t in per_task if t["kernel"] == "tensor"]
+        dw = [t for t in per_task if t["kernel"] == "depthwise"]
+        t_tens, t_dw = sum(t["ms"] for t in tens), sum(t["ms"] for t in dw)
+        if t_dw > t_tens and dw:
+            gb = sum(t["bytes"] for t in dw) / 1e9
+            ach = gb / (t_dw * 1e-3)
+            roof = {"kernel": "depthwise3x3_kernel", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "launches_per_step": len(dw), "ms_per_step": t_dw}
+        elif tens:
+            tf = sum(t["flops"] for t in tens) / 1e12
+            ach = tf / (t_tens * 1e-3)
+            roof = {"kernel": "conv_tc_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained bf16 GEMM)", "launches_per_step": len(tens),
+                    "ms_per_step": t_tens}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        a = argparse.Namespace(steps=1, warmup=0)
+        import oracle  # the CPU-baseline leg is the one place the benchmark may run the oracle
+        sample = {"resnet18": 16, "mobilenet_v2": 32, "vgg16_cifar": 96}[table_name]
+        pw, _ = oracle.prune_model(table, weights)
+        xs = wl.model_input(table, sample)
+        t0 = time.perf_counter()
+        oracle.model_ref(table, pw, xs, matched=True)
+        dt = time.perf_counter() - t0
+        cpu = {"value": sample / dt, "unit": "images/s", "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": "%d images of %s, one pass, %.1f s" % (sample, cfg["workload"], dt)}
+
+    images = batch * world * args.steps
+    in_bytes = x_host.numel() * 4
+    out_bytes = logits_host.numel() * 4
+    line = {"metric": "pruned_model_images_per_s", "value": images / (ms * 1e-3), "unit": "images/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
+            "tflops": net.flops() * world * args.steps / (ms * 1e-3) / 1e12,
+            "e2e": {"value": images / (ms_e2e * 1e-3), "unit": "images/s", "h2d_bytes_per_step": in_bytes,
+                    "d2h_bytes_per_step": out_bytes, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": net.model.launches * args.steps, "launches_per_step": net.model.launches,
+            "cuda_graph": use_graph, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
+            "prepare_ms": prepare_ms, "prepare_first_ms": prepare_first_ms,
+            "tasks": per_task}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def net_task_times(cp, net, table, x, reps=5):
+    """Times every conv task with CUDA events on the launching stream inside eager passes of the
+    whole model, one launch per task per pass, so that each task sees the cache state its
+    predecessor left (no artificial L2 warmth from repeating one task).  Median over the passes."""
+    import torch
+    stream = torch.cuda.current_stream()
+    bufs, times, infos = {}, {}, {}
+    for rep in range(reps + 1):                       # the first pass allocates and warms up
+        acts = {"x": cp.cprune_cast_input(x, bufs.get("x"))}
+        bufs["x"] = acts["x"]
+        for l in table["layers"]:
+            kind = l["kind"]
+            a = acts[l["in"]]
+            if kind == "conv":
+                plan = net.plans[l["name"]]
+                wp, bp = net.packed[l["name"]]
+                res = acts[l["res"]] if l.get("res") else None
+                if l["name"] not in bufs:
+                    bufs[l["name"]] = (torch.empty((plan.N, plan.out_h, plan.out_w, plan.k_pad), dtype=torch.bfloat16,
+                                                   device=x.device),
+                                       torch.empty(max(plan.workspace_bytes, 16), dtype=torch.uint8, device=x.device))
+                y, ws = bufs[l["name"]]
+                s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s.record(stream)
+                cp.cprune_task_run(plan, a, wp, bp, res, y, ws)
+                e.record(stream)
+                if rep > 0:
+                    times.setdefault(l["name"], []).append((s, e))
+                infos[l["name"]] = plan.info
+                acts[l["out"]] = y
+            elif kind == "maxpool":
+                acts[l["out"]] = cp.cprune_maxpool(a, a.shape[-1], l["k"], l["stride"], l["pad"])
+            elif kind == "gap":
+                acts[l["out"]] = cp.cprune_global_avgpool(a, a.shape[-1])
+            elif kind == "flatten":
+                acts[l["out"]] = a
+            elif kind == "fc":
+                break
+    torch.cuda.synchronize()
+    out = []
+    for name, evs in times.items():
+        ms = float(np.median([s.elapsed_time(e) for s, e in evs]))
+        i = infos[name]
+        out.append({"name": name, "kernel": cp.KERNEL_NAMES[i["kernel"]], "C": i["C"], "K": i["K"],
+                    "HW": [i["H"], i["W"]], "R": i["R"], "stride": i["stride"], "ms": ms, "flops": i["flops"],
+                    "bytes": i["algorithmic_bytes"], "tflops": i["flops"] / ms / 1e9,
+                    "gbs": i["algorithmic_bytes"] / ms / 1e6, "tile_n": i["tile_n"], "tiles": i["tiles_m"] * i["tiles_n"]})
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -27,6 +27,7 @@ struct cprune_model {
     const float *graph_x = nullptr;
     float *graph_logits = nullptr;
     cudaStream_t graph_stream = nullptr;
+    cudaStream_t capture_stream = nullptr;   // private stream the launch sequence is recorded on
 };
 
 namespace cprune {
@@ -172,10 +173,13 @@ cprune_status cprune_model_run(cprune_model *m, const float *x, float *logits, i
     // kernel attributes outside of any capture), then record the same sequence for later replays
     cprune_status s = enqueue(m, x, logits, st);
     if (s != CPRUNE_OK) return s;
+    // the caller's stream may be the legacy default stream, which cannot be captured: record on a
+    // private stream and replay the graph on the caller's
+    if (!m->capture_stream) CPRUNE_CUDA_CHECK(cudaStreamCreateWithFlags(&m->capture_stream, cudaStreamNonBlocking));
     cudaGraph_t graph = nullptr;
-    CPRUNE_CUDA_CHECK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-    s = enqueue(m, x, logits, st);
-    cudaError_t e = cudaStreamEndCapture(st, &graph);
+    CPRUNE_CUDA_CHECK(cudaStreamBeginCapture(m->capture_stream, cudaStreamCaptureModeThreadLocal));
+    s = enqueue(m, x, logits, m->capture_stream);
+    cudaError_t e = cudaStreamEndCapture(m->capture_stream, &graph);
     if (s != CPRUNE_OK) { if (graph) cudaGraphDestroy(graph); return s; }
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
     e = cudaGraphInstantiate(&m->exec, graph, 0);
@@ -211,6 +215,7 @@ int cprune_model_launches(const cprune_model *m) { return m ? m->launches : 0; }
 cprune_status cprune_model_destroy(cprune_model *m) {
     if (!m) return CPRUNE_ERR_INVALID_ARG;
     if (m->exec) cudaGraphExecDestroy(m->exec);
+    if (m->capture_stream) cudaStreamDestroy(m->capture_stream);
     if (m->arena) cudaFree(m->arena);
     if (m->workspace) cudaFree(m->workspace);
     delete m;
