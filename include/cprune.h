@@ -84,6 +84,29 @@ cprune_status cprune_select_filters(const float *w, const float *b, int K, int C
                                     int32_t *kept_idx, float *w_out, float *b_out, float *w_next_out,
                                     void *workspace, size_t workspace_bytes, void *stream);
 
+/* The same selection for callers that must not allocate device memory and have no scratch buffer
+ * to hand over: code that runs where a cudaMalloc would stall or is forbidden (inside a latency-
+ * critical serving loop, under a framework that has already claimed the whole device, in a process
+ * whose memory budget is fixed at start-up).  (The paper has no counterpart to this entry point; it
+ * exists for the library's users.)  It takes the arguments of cprune_select_filters without the
+ * workspace and keeps the per-filter norms and keep flags in a fixed buffer that lives inside the
+ * library image: 48 KiB of device memory on every GPU that loads the library, held until the
+ * process exits.  The caller still provides every input and output buffer.
+ *   - K must not exceed CPRUNE_SELECT_STATIC_MAX_FILTERS; a larger K returns
+ *     CPRUNE_ERR_WORKSPACE_TOO_SMALL and launches nothing.
+ *   - It calls no allocating routine (no cudaMalloc / cudaFree).  The first call on each device
+ *     looks up the buffer's device address once; make that first call outside any stream capture.
+ *   - All calls on a device share the one buffer, which keeps whatever the previous call left.
+ *     Every entry a call reads it has written first, so nothing needs clearing, but two calls
+ *     whose kernels overlap on the GPU (different streams, no ordering between them) race on it:
+ *     order them on one stream or with events.
+ * Results are bit-identical to cprune_select_filters. */
+#define CPRUNE_SELECT_STATIC_MAX_FILTERS 4096
+cprune_status cprune_select_filters_static(const float *w, const float *b, int K, int C, int R, int S, int keep_k,
+                                           const float *w_next, int K2, int R2, int S2, int next_is_depthwise,
+                                           int32_t *kept_idx, float *w_out, float *b_out, float *w_next_out,
+                                           void *stream);
+
 /* Row gather out[j][:] = in[idx[j]][:] (inner floats per row) and column gather
  * out[o][j][:] = in[o][idx[j]][:] for further consumers of the same kept_idx (a depthwise layer's
  * bias, the project layer behind a depthwise layer, the first FC layer).  All pointers device. */

@@ -23,7 +23,7 @@ OP_CONV, OP_MAXPOOL, OP_GAP, OP_FC = 1, 2, 3, 4
 # every symbol include/cprune.h declares
 EXPORTS = [
     "cprune_status_string", "cprune_last_cuda_error", "cprune_padded_channels", "cprune_select_workspace_bytes",
-    "cprune_select_filters", "cprune_gather_rows", "cprune_gather_columns", "cprune_task_plan", "cprune_plan_query",
+    "cprune_select_filters", "cprune_select_filters_static", "cprune_gather_rows", "cprune_gather_columns", "cprune_task_plan", "cprune_plan_query",
     "cprune_plan_release", "cprune_cache_clear", "cprune_cache_stats", "cprune_pack_weights", "cprune_task_run",
     "cprune_cast_input", "cprune_widen_output", "cprune_maxpool", "cprune_global_avgpool", "cprune_fc_pack",
     "cprune_fc", "cprune_model_create", "cprune_model_run", "cprune_model_tensor", "cprune_model_copy_tensor", "cprune_model_launches",
@@ -74,6 +74,8 @@ def lib():
         L.cprune_select_filters.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_int,
                                             c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                             c_size_t, c_void_p]
+        L.cprune_select_filters_static.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_int,
+                                                   c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.cprune_gather_rows.argtypes = [c_void_p, c_int, c_size_t, c_void_p, c_int, c_void_p, c_void_p]
         L.cprune_gather_columns.argtypes = [c_void_p, c_int, c_int, c_size_t, c_void_p, c_int, c_void_p, c_void_p]
         L.cprune_task_plan.argtypes = [c_int] * 10 + [POINTER(TaskOpts), POINTER(c_void_p)]
@@ -155,6 +157,31 @@ def cprune_select_filters(w, keep_k, b=None, w_next=None, next_is_depthwise=Fals
                                      _ptr(workspace), workspace.numel(), _stream(stream))
     _check(st, "cprune_select_filters")
     return kept, w_out, b_out, wn_out
+
+
+SELECT_STATIC_MAX_FILTERS = 4096
+
+
+def cprune_select_filters_static(w, keep_k, kept_idx, w_out, b=None, b_out=None, w_next=None, w_next_out=None,
+                                 next_is_depthwise=False, stream=None):
+    """Selection without any device allocation: the caller passes every output buffer and the library
+    uses its built-in scratch (at most SELECT_STATIC_MAX_FILTERS filters).  For callers that cannot
+    allocate: serving loops, processes with a fixed memory budget.  Calls that overlap on the GPU race
+    on the shared scratch, so keep them ordered on one stream."""
+    w = _dev_f32(w)
+    K, C, R, S = w.shape
+    K2 = R2 = S2 = 0
+    if w_next is not None:
+        w_next = _dev_f32(w_next)
+        if next_is_depthwise:
+            _, _, R2, S2 = w_next.shape
+        else:
+            K2, _, R2, S2 = w_next.shape
+    st = lib().cprune_select_filters_static(_ptr(w), _ptr(b), K, C, R, S, int(keep_k), _ptr(w_next), K2, R2, S2,
+                                            1 if next_is_depthwise else 0, _ptr(kept_idx), _ptr(w_out), _ptr(b_out),
+                                            _ptr(w_next_out), _stream(stream))
+    _check(st, "cprune_select_filters_static")
+    return kept_idx, w_out, b_out, w_next_out
 
 
 def cprune_gather_rows(t, idx, stream=None):

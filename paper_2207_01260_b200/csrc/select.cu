@@ -132,6 +132,30 @@ __global__ void gather_cols_kernel(const float *__restrict__ in, int outer, int 
     }
 }
 
+// Scratch of the allocation-free entry point: norms (int64) followed by keep flags (int32) for up
+// to CPRUNE_SELECT_STATIC_MAX_FILTERS filters.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a pointer that a kernel may be given.
+constexpr size_t STATIC_NORM_BYTES = (size_t)CPRUNE_SELECT_STATIC_MAX_FILTERS * sizeof(long long);
+constexpr size_t STATIC_KEEP_BYTES = (size_t)CPRUNE_SELECT_STATIC_MAX_FILTERS * sizeof(int);
+static __device__ __align__(256) unsigned char g_select_scratch[STATIC_NORM_BYTES + STATIC_KEEP_BYTES];
+
+// Device address of g_select_scratch on the current device, looked up once per device.
+static cprune_status select_scratch_address(unsigned char **out) {
+    static std::mutex mu;
+    static unsigned char *ptrs[64] = {nullptr};
+    int dev = 0;
+    CPRUNE_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CPRUNE_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        unsigned char *p = nullptr;
+        CPRUNE_CUDA_CHECK(cudaGetSymbolAddress((void **)&p, g_select_scratch));
+        ptrs[dev] = p;
+    }
+    *out = ptrs[dev];
+    return CPRUNE_OK;
+}
+
 static int grid_for(size_t total, int threads) {
     size_t g = (total + threads - 1) / threads;
     if (g < 1) g = 1;
@@ -216,6 +240,28 @@ cprune_status cprune_select_filters(const float *w, const float *b, int K, int C
     if (!status) return cuda_fail(cudaGetLastError(), "status word");
     long long *norms = (long long *)workspace;
     int *keep = (int *)((char *)workspace + align_up((size_t)K * sizeof(long long), 256));
+    return select_launch(w, b, K, C, R, S, keep_k, w_next, K2, R2, S2, next_is_depthwise, kept_idx, w_out, b_out,
+                         w_next_out, norms, keep, status, (cudaStream_t)stream);
+}
+
+cprune_status cprune_select_filters_static(const float *w, const float *b, int K, int C, int R, int S, int keep_k,
+                                           const float *w_next, int K2, int R2, int S2, int next_is_depthwise,
+                                           int32_t *kept_idx, float *w_out, float *b_out, float *w_next_out,
+                                           void *stream) {
+    if (!w || !kept_idx || !w_out || K <= 0 || C <= 0 || R <= 0 || S <= 0) return CPRUNE_ERR_INVALID_ARG;
+    if (keep_k < 1 || keep_k > K) return CPRUNE_ERR_INVALID_ARG;
+    if (b && !b_out) return CPRUNE_ERR_INVALID_ARG;
+    if (w_next && (!w_next_out || R2 <= 0 || S2 <= 0 || (!next_is_depthwise && K2 <= 0))) return CPRUNE_ERR_INVALID_ARG;
+    if ((size_t)C * R * S > 8192) return CPRUNE_ERR_UNSUPPORTED;
+    if (K > CPRUNE_SELECT_STATIC_MAX_FILTERS) return CPRUNE_ERR_WORKSPACE_TOO_SMALL;   // beyond the fixed buffer
+    unsigned char *scratch = nullptr;
+    cprune_status st = select_scratch_address(&scratch);
+    if (st != CPRUNE_OK) return st;
+    int *status = device_status_word();
+    if (!status) return cuda_fail(cudaGetLastError(), "status word");
+    // every norm and keep flag below K is written before it is read, so stale contents are harmless
+    long long *norms = (long long *)scratch;
+    int *keep = (int *)(scratch + STATIC_NORM_BYTES);
     return select_launch(w, b, K, C, R, S, keep_k, w_next, K2, R2, S2, next_is_depthwise, kept_idx, w_out, b_out,
                          w_next_out, norms, keep, status, (cudaStream_t)stream);
 }
