@@ -115,7 +115,11 @@ def main():
     ap.add_argument("--workload", default="resnet18", choices=sorted(WORKLOADS))
     ap.add_argument("--no-graph", action="store_true", help="enqueue every launch from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--task", default=None,
+                    help="time ONE conv task instead of a model: N,C,H,W,K,R,stride,pad[,groups[,act[,residual]]]")
     args = ap.parse_args()
+    if args.task:
+        return task_bench(args)
     table_name, batch = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -271,6 +275,58 @@ def main():
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def task_bench(args):
+    """One conv task, timed with CUDA events over `steps` launches that rotate through enough
+    distinct (x, y) buffer sets to exceed twice the L2 size (cold), and again on one set (warm)."""
+    import torch
+
+    import paper_2207_01260_b200 as cp
+    import workloads as wl
+    f = args.task.split(",")
+    N, C, H, W, K, R, stride, pad = [int(v) for v in f[:8]]
+    groups = int(f[8]) if len(f) > 8 else 1
+    act = f[9] if len(f) > 9 else "relu"
+    residual = len(f) > 10 and f[10] == "1"
+    torch.cuda.set_device(0)
+    plan = cp.cprune_task_plan(N, C, H, W, K, R, R, stride, pad, groups, act, residual)
+    i = plan.info
+    x, w, b, res = wl.conv_task_tensors(7, N, C, H, W, K, R, R, groups, residual, i["P"], i["Q"])
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    wp, bp = cp.cprune_pack_weights(plan, dev(w), dev(b))
+    xb = cp.cprune_cast_input(dev(x))
+    rb = cp.cprune_cast_input(dev(res)) if residual else None
+    set_bytes = xb.numel() * 2 + N * i["out_h"] * i["out_w"] * i["k_pad"] * 2
+    nsets = int(max(1, min(64, -(-2 * 126e6 // set_bytes))))
+    xs = [xb] + [xb.clone() for _ in range(nsets - 1)]
+    ys = [torch.empty((N, i["out_h"], i["out_w"], i["k_pad"]), dtype=torch.bfloat16, device="cuda") for _ in range(nsets)]
+    ws = torch.empty(max(i["workspace_bytes"], 16), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def timed(rotate):
+        for j in range(max(args.warmup, 3)):
+            cp.cprune_task_run(plan, xs[j % nsets if rotate else 0], wp, bp, rb, ys[j % nsets if rotate else 0], ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for j in range(args.steps):
+            cp.cprune_task_run(plan, xs[j % nsets if rotate else 0], wp, bp, rb, ys[j % nsets if rotate else 0], ws)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    ms_cold, ms_warm = timed(True), timed(False)
+    cp.cprune_poll_device_status()
+    peaks = measured_peaks()
+    line = {"metric": "conv_task_tflops", "task": args.task, "kernel": cp.KERNEL_NAMES[i["kernel"]],
+            "ms_cold": ms_cold, "ms_warm": ms_warm, "tflops_cold": i["flops"] / ms_cold / 1e9,
+            "tflops_warm": i["flops"] / ms_warm / 1e9, "gbs_cold": i["algorithmic_bytes"] / ms_cold / 1e6,
+            "frac_tensor_peak": i["flops"] / ms_cold / 1e9 / peaks["bf16_tflops"],
+            "frac_hbm_peak": i["algorithmic_bytes"] / ms_cold / 1e6 / peaks["hbm_gbs"],
+            "buffer_sets": nsets, "tile_n": i["tile_n"], "tiles": i["tiles_m"] * i["tiles_n"], "stages": i["stages"],
+            "steps": args.steps, "padded_flops_ratio": i["padded_flops"] / i["flops"]}
+    print(json.dumps(line))
 
 
 def net_task_times(cp, net, table, x, reps=5):
