@@ -1,23 +1,29 @@
 // Dense conv task as an implicit GEMM on the sm_100a tensor cores (paper Sec. 3.4: a task is
 // Conv2d + folded BatchNorm + activation; Sec. 3.5: the filter count K is whatever pruning left).
 //
-//   D[m][k] = sum over (r, s, c) of  X[pixel m shifted by tap (r,s)][c] * Wt[k][r][s][c]
-//   m = output pixel (n, p, q) linearised,  GEMM-M = N*P*Q,  GEMM-N = K,  GEMM-K = R*S*C
+//   D[pixel][k] = sum over (r, s, c) of  X[pixel shifted by tap (r,s)][c] * Wt[k][r][s][c]
+//   GEMM-M = N*P*Q output pixels,  GEMM-N = K filters,  GEMM-K = R*S*C
 //
 // One persistent CTA per SM, 192 threads, three roles:
-//   warp 0      producer: per (tap, 64-channel block) one im2col TMA load of 128 pixels x 64
+//   warp 0      producer: per (tap, 64-channel block) one im2col-mode TMA load of PT pixels x 64
 //               channels of the activation tensor (zero fill for the padding border and for
-//               channels beyond c_pad) and one tiled TMA load of BN filters x 64 channels,
-//               both into 128-byte-swizzled shared memory, completion on an mbarrier;
-//   warp 1      issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction, bf16 x bf16 ->
+//               channels beyond c_pad) and one tiled TMA load of FT filters x 64 channels, both
+//               into 128-byte-swizzled shared memory, completion on an mbarrier;
+//   warp 1      one elected lane issues tcgen05.mma (K = 16 per instruction, bf16 x bf16 ->
 //               float32) with the accumulator in tensor memory; two accumulator buffers so
 //               that the epilogue of one tile overlaps the main loop of the next;
-//   warps 2..5  epilogue: tcgen05.ld the accumulator, add bias (+ residual), activation,
-//               convert to bf16 and store NHWC rows.
-// Odd channel counts: C is padded to a multiple of 8 in memory, the last channel block issues
-// only ceil(remaining/16) MMAs; K is covered by tiles_n tiles of BN (a multiple of 16).
-// Every wait is bounded: when a limit expires the CTA raises STATUS_TIMEOUT in the device status
-// word, all roles leave their loops, tensor memory is released and the kernel returns.
+//   warps 2..5  epilogue: tcgen05.ld the accumulator, bias (+ residual), activation, bf16,
+//               write 16-filter-wide sub-tiles into swizzled shared memory, TMA-store them to
+//               the NHWC output (the store clips rows beyond the last pixel and filters beyond
+//               k_pad by itself).
+// An MMA instruction costs about the same for any N up to 256, so the plan picks the orientation
+// that keeps N large:
+//   ORIENT_PIX  (K > 128): MMA-M = 128 pixels,  MMA-N = BN filters (multiple of 16, <= 256);
+//   ORIENT_FILT (K <= 128): MMA-M = 128 filter rows (zero rows above K), MMA-N = 256 pixels.
+// Odd channel counts: C is padded to a multiple of 8 in memory and the last channel block issues
+// only ceil(remaining/16) MMAs.  Every wait is bounded: when a limit expires the CTA raises
+// STATUS_TIMEOUT in the device status word, all roles leave their loops, tensor memory is
+// released and the kernel returns.
 #include <cuda.h>
 
 #include <cstring>
@@ -29,29 +35,43 @@
 namespace cprune {
 
 constexpr int TC_THREADS = 192;
-constexpr int BM = 128;            // pixels per tile (MMA M)
 constexpr int BK = 64;             // channels per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;    // column offset of the second accumulator buffer
 constexpr int MAX_STAGES = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 1LL << 31;   // about a second
+constexpr int ORIENT_PIX = 0, ORIENT_FILT = 1;
+constexpr int SUB = 16;            // filters per staged sub-tile (32-byte rows, 32-byte swizzle)
+constexpr int CTRL_BYTES = 2048;   // barriers, flags, bias vector
+constexpr int GROUP_BYTES = 16384; // one staging buffer (see the kernel)
 
 struct TcParams {
     long long M;
     int P, Q, stride, pad, R, S;
     int cblks;         // ceil(c_pad / 64)
     int ksteps_last;   // 16-channel MMA steps in the last channel block
-    int BN, tiles_m, tiles_n, k_pad, stages, act;
+    int PT, FT;        // pixels and filters per tile
+    int tiles_m, tiles_n, k_pad, stages, act;
+    int staging_bufs;  // 1 or 2 staging buffers of PT_GROUP x 64 bf16
     const float *bias;
     const __nv_bfloat16 *res;
-    __nv_bfloat16 *y;
     int *status;
 };
 
 // ------------------------------------------------------------------------------------------ PTX
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+        "elect.sync rx|px, %1;\n\t"
+        "selp.u32 %0, 1, 0, px;\n\t}"
+        : "=r"(pred)
+        : "r"(0xFFFFFFFFu));
+    return pred;
+}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -74,14 +94,15 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 
-// Bounded wait.  Returns false when the limit expired here or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+// Bounded wait.  Returns false when the limit expired here or (if watch_abort) another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          bool watch_abort = true) {
     for (int i = 0; i < 64; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
+        if (watch_abort && *abort_flag) return false;
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
             atomicOr(status, STATUS_TIMEOUT);
             *abort_flag = 1;
@@ -107,6 +128,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         : "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 :
+                 : "l"(map), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
@@ -157,24 +191,38 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 
+// Byte offset of (row, 16-byte half h) in a staged sub-tile of 32-byte rows under the 32-byte
+// swizzle (address bit 4 is XORed with bit 7, i.e. with bit 2 of the row).
+__device__ __forceinline__ uint32_t sub_off(int row, int h) { return (uint32_t)(row * 32 + ((h ^ ((row >> 2) & 1)) << 4)); }
+
 // ---------------------------------------------------------------------------------------- kernel
 
+template <int ORIENT>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const TcParams p) {
+conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+               const __grid_constant__ CUtensorMap tm_y, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     uint8_t *smem = smem_raw + (base - raw);
-    const int stage_bytes = A_STAGE_BYTES + p.BN * BK * 2;
-    uint8_t *ctrl = smem + (size_t)p.stages * stage_bytes;
-    const uint32_t bar0 = base + (uint32_t)p.stages * stage_bytes;
-    // barrier slots (8 bytes each): full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2]
-    auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
-    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + 2 + a); };
-    uint32_t *tmem_slot = (uint32_t *)(ctrl + 8 * (2 * MAX_STAGES + 4));
-    volatile int *abort_flag = (volatile int *)(ctrl + 8 * (2 * MAX_STAGES + 4) + 4);
+    const int x_bytes = p.PT * BK * 2;                     // pixel operand of one stage
+    const int stage_bytes = x_bytes + p.FT * BK * 2;
+    // staging buffers, each one group of sub-tiles [rows][16 filters] bf16:
+    //   ORIENT_PIX:  128 pixels x 64 filters  = 4 sub-tiles of 4 KB
+    //   ORIENT_FILT:  64 pixels x 128 filters = 8 sub-tiles of 2 KB
+    constexpr int GROUP_ROWS = ORIENT == ORIENT_PIX ? 128 : 64;
+    constexpr int SUB_BYTES = GROUP_ROWS * SUB * 2;
+    const uint32_t staging0 = base + (uint32_t)p.stages * stage_bytes;
+    const uint32_t ctrl0 = staging0 + (uint32_t)p.staging_bufs * GROUP_BYTES;
+    uint8_t *ctrl = smem + (ctrl0 - base);
+    // barrier slots (8 bytes each): full[8], empty[8], tfull[2], tempty[2], epi[1]
+    auto full_bar = [&](int s) { return ctrl0 + 8u * s; };
+    auto empty_bar = [&](int s) { return ctrl0 + 8u * (MAX_STAGES + s); };
+    auto tfull_bar = [&](int a) { return ctrl0 + 8u * (2 * MAX_STAGES + a); };
+    auto tempty_bar = [&](int a) { return ctrl0 + 8u * (2 * MAX_STAGES + 2 + a); };
+    const uint32_t epi_bar = ctrl0 + 8u * (2 * MAX_STAGES + 4);
+    uint32_t *tmem_slot = (uint32_t *)(ctrl + 8 * (2 * MAX_STAGES + 5));
+    volatile int *abort_flag = (volatile int *)(ctrl + 8 * (2 * MAX_STAGES + 5) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -187,6 +235,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             mbar_init(tfull_bar(a), 1);
             mbar_init(tempty_bar(a), 4);
         }
+        mbar_init(epi_bar, 4);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -209,7 +258,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
-            const long long m0 = (long long)mt * BM;
+            const long long m0 = (long long)mt * p.PT;
             const int n_img = (int)(m0 / PQ);
             const int rem = (int)(m0 - (long long)n_img * PQ);
             const int p0 = rem / p.Q, q0 = rem - p0 * p.Q;
@@ -217,13 +266,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             for (int r = 0; r < p.R && ok; ++r)
                 for (int s = 0; s < p.S && ok; ++s)
                     for (int cb = 0; cb < p.cblks; ++cb) {
-                        ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
+                        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                         if (!ok) break;
-                        if (lane == 0) {
-                            const uint32_t a_dst = base + (uint32_t)stage * stage_bytes;
+                        if (elect_one()) {
+                            const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
                             mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
-                            tma_load_im2col(a_dst, &tm_a, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
-                            tma_load_3d(a_dst + A_STAGE_BYTES, &tm_b, full_bar(stage), cb * BK, r * p.S + s, nt * p.BN);
+                            tma_load_im2col(x_dst, &tm_x, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
+                            tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), cb * BK, r * p.S + s, nt * p.FT);
                         }
                         __syncwarp();
                         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -231,87 +280,204 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issue
-        // instruction descriptor: D float32, A and B bf16, both K-major, N = BN, M = 128
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        // instruction descriptor: D float32, A and B bf16, both K-major, M = 128, N = filters or pixels
+        const int mma_n = ORIENT == ORIENT_PIX ? p.FT : p.PT;
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         int stage = 0, acc = 0;
         uint32_t phase = 0, acc_phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status);
+            ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_STRIDE);
             uint32_t accumulate = 0;
             for (int tap = 0; tap < p.R * p.S && ok; ++tap)
                 for (int cb = 0; cb < p.cblks; ++cb) {
-                    ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status);
+                    ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag, p.status));
                     if (!ok) break;
-                    tc_fence_after();
-                    if (lane == 0) {
-                        const uint32_t a_addr = base + (uint32_t)stage * stage_bytes;
-                        const uint64_t da = smem_desc_sw128(a_addr);
-                        const uint64_t db = smem_desc_sw128(a_addr + A_STAGE_BYTES);
-                        const int nk = (cb == p.cblks - 1) ? p.ksteps_last : BK / 16;
+                    const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
+                    const uint64_t dx = smem_desc_sw128(x_addr);
+                    const uint64_t dw = smem_desc_sw128(x_addr + x_bytes);
+                    const int nk = (cb == p.cblks - 1) ? p.ksteps_last : BK / 16;
+                    if (elect_one()) {
                         for (int kk = 0; kk < nk; ++kk) {
                             // 16 channels = 32 bytes further along the swizzled row: +2 in 16-byte units
-                            umma_bf16(d_tmem, da + (uint64_t)(2 * kk), db + (uint64_t)(2 * kk), idesc, accumulate);
+                            if (ORIENT == ORIENT_PIX)
+                                umma_bf16(d_tmem, dx + (uint64_t)(2 * kk), dw + (uint64_t)(2 * kk), idesc, accumulate);
+                            else
+                                umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dx + (uint64_t)(2 * kk), idesc, accumulate);
                             accumulate = 1;
                         }
                         umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
                     }
+                    accumulate = 1;
                     __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
-            if (ok && lane == 0) umma_commit(tfull_bar(acc));
+            if (ok && elect_one()) umma_commit(tfull_bar(acc));
             __syncwarp();
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     } else {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int row = quarter * 32 + lane;
+        const int et = (warp - 2) * 32 + lane;         // 0..127 among the epilogue threads
+        const int trow = quarter * 32 + lane;          // accumulator row (pixel or filter) of this thread
+        const bool store_thread = et == 0;
         int acc = 0;
-        uint32_t acc_phase = 0;
+        uint32_t acc_phase = 0, epi_phase = 0;
+        uint32_t group_counter = 0;                    // staged groups so far (selects the buffer)
         bool ok = true;
+        // Bounded barrier among the four epilogue warps (one arrival per warp).  Per staged group:
+        // everyone writes buffer g%2, the store thread makes sure every earlier store has been read
+        // out of shared memory, all meet here, then the store thread issues the stores of group g.
+        // Buffer g%2 was last used by group g-2, whose store was confirmed read before barrier g-1.
+        auto epi_sync = [&]() {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(epi_bar);
+            bool r = __all_sync(0xffffffffu, mbar_wait(epi_bar, epi_phase, abort_flag, p.status, false));
+            epi_phase ^= 1u;
+            return r;
+        };
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
-            const long long m = (long long)mt * BM + row;
-            ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
+            const long long m0 = (long long)mt * p.PT;
+            const int k_base = nt * p.FT;
+            // the epilogue ignores the abort flag: all four warps must take the same decisions,
+            // and they all watch the same barriers
+            ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, false));
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * ACC_STRIDE);
-            const bool row_ok = m < p.M;
-            __nv_bfloat16 *yrow = p.y + (size_t)(row_ok ? m : 0) * p.k_pad;
-            const __nv_bfloat16 *rrow = p.res ? p.res + (size_t)(row_ok ? m : 0) * p.k_pad : nullptr;
-            for (int c0 = 0; c0 < p.BN; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld16(t_row + (uint32_t)c0, v);
-                tmem_ld_wait();
-                const int kg = nt * p.BN + c0;
+
+            if (ORIENT == ORIENT_PIX) {
+                // rows = pixels, columns = filters; groups of 64 filters
+                const long long m = m0 + trow;
+                const bool row_ok = m < p.M;
+                const bool has_res = p.res != nullptr && row_ok;
+                const int groups = (p.FT + 63) / 64;
+                for (int g = 0; g < groups && ok; ++g) {
+                    uint8_t *buf_ptr = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES;
+                    const uint32_t buf = staging0 + (group_counter & 1u) * GROUP_BYTES;
+                    const int cg = g * 64;                       // first filter column of the group
+                    // residual of this group: 64 filters = 128 contiguous bytes of the thread's row
+                    bf16x8 rv[8];
+                    if (has_res) {
+                        const __nv_bfloat16 *rrow = p.res + (size_t)m * p.k_pad + k_base + cg;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int k0 = kg + half * 8;
-                    if (row_ok && k0 < p.k_pad) {
-                        float f[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[half * 8 + j]) + __ldg(p.bias + k0 + j);
-                        if (rrow) {
-                            float rf[8];
-                            unpack8(ldg8((const bf16x8 *)(rrow + k0)), rf);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) f[j] += rf[j];
-                        }
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], p.act);
-                        *(bf16x8 *)(yrow + k0) = pack8(f);
+                        for (int j = 0; j < 8; ++j)
+                            if (k_base + cg + j * 8 < p.k_pad) rv[j] = ldg8((const bf16x8 *)(rrow + j * 8));
                     }
+                    uint32_t v[64];
+#pragma unroll
+                    for (int sb = 0; sb < 4; ++sb)
+                        if (cg + sb * SUB < p.FT) tmem_ld16(t_row + (uint32_t)(cg + sb * SUB), v + sb * 16);
+                    tmem_ld_wait();
+                    if (g == groups - 1) {               // accumulator fully read: hand it back to the MMA warp
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty_bar(acc));
+                    }
+#pragma unroll
+                    for (int sb = 0; sb < 4; ++sb) {
+                        const int c0 = cg + sb * SUB;
+                        if (c0 < p.FT) {
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float f[8];
+                                const float4 b0 = __ldg((const float4 *)(p.bias + k_base + c0 + h * 8));
+                                const float4 b1 = __ldg((const float4 *)(p.bias + k_base + c0 + h * 8 + 4));
+                                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[sb * 16 + h * 8 + j]) + bb[j];
+                                if (has_res && k_base + c0 + h * 8 < p.k_pad) {
+                                    float rf[8];
+                                    unpack8(rv[sb * 2 + h], rf);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) f[j] += rf[j];
+                                }
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], p.act);
+                                *(bf16x8 *)(buf_ptr + sb * SUB_BYTES + sub_off(trow, h)) = pack8(f);
+                            }
+                        }
+                    }
+                    fence_async_smem();
+                    if (store_thread) tma_store_wait_read<0>();
+                    ok = epi_sync();
+                    if (!ok) break;
+                    if (store_thread) {
+                        for (int sb = 0; sb < 4; ++sb) {
+                            const int c0 = cg + sb * SUB;
+                            if (c0 < p.FT && k_base + c0 < p.k_pad)
+                                tma_store_2d(&tm_y, buf + sb * SUB_BYTES, k_base + c0, (int)m0);
+                        }
+                        tma_store_commit();
+                    }
+                    ++group_counter;
+                }
+            } else {
+                // rows = filters, columns = pixels; groups of 64 pixels
+                const int k = trow;                       // this thread's filter
+                const bool k_ok = k < p.k_pad;
+                const float bias = k_ok ? __ldg(p.bias + k) : 0.f;
+                const int n_sub = (p.k_pad + SUB - 1) / SUB;       // sub-tiles that hold real filters
+                const bool warp_has_work = quarter * 32 < p.k_pad; // all 32 filters of this warp may be padding
+                const int groups = p.PT / 64;
+                const int hk = (k >> 3) & 1;
+                for (int g = 0; g < groups && ok; ++g) {
+                    uint8_t *dst = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 4) * SUB_BYTES + (k & 7) * 2;
+                    const uint32_t buf = staging0 + (group_counter & 1u) * GROUP_BYTES;
+                    const long long mg = m0 + g * 64;
+                    if (warp_has_work) {
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            // residual values of 32 pixels for this filter, all loads in flight together
+                            unsigned short rr[32];
+                            const bool has_res = p.res != nullptr && k_ok;
+                            if (has_res) {
+                                const unsigned short *rp = (const unsigned short *)p.res + (size_t)(mg + half * 32) * p.k_pad + k;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    rr[j] = (mg + half * 32 + j < p.M) ? __ldg(rp + (size_t)j * p.k_pad) : (unsigned short)0;
+                            }
+                            uint32_t v[32];
+                            tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32), v);
+                            tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32 + 16), v + 16);
+                            tmem_ld_wait();
+                            if (k_ok) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    const int px = half * 32 + j;
+                                    float f = __uint_as_float(v[j]) + bias;
+                                    if (has_res) f += __uint_as_float((uint32_t)rr[j] << 16);
+                                    f = apply_act(f, p.act);
+                                    *(__nv_bfloat16 *)(dst + sub_off(px, hk)) = __float2bfloat16_rn(f);
+                                }
+                            }
+                        }
+                    }
+                    if (g == groups - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty_bar(acc));
+                    }
+                    fence_async_smem();
+                    if (store_thread) tma_store_wait_read<0>();
+                    ok = epi_sync();
+                    if (!ok) break;
+                    if (store_thread) {
+                        for (int sb = 0; sb < n_sub; ++sb)
+                            tma_store_2d(&tm_y, buf + sb * SUB_BYTES, sb * SUB, (int)mg);
+                        tma_store_commit();
+                    }
+                    ++group_counter;
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        if (store_thread) tma_store_wait_all();          // staged data must be read before the CTA's memory goes away
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -358,67 +524,80 @@ static cprune_status load_driver_entry_points() {
     return CPRUNE_OK;
 }
 
-static int smem_for(int stages, int BN) {
-    return 1024 /* alignment slack */ + stages * (A_STAGE_BYTES + BN * BK * 2) + 8 * (2 * MAX_STAGES + 4) + 16;
+static int smem_for(int stages, int PT, int FT, int staging_bufs, int group_rows) {
+    (void)group_rows;
+    return 1024 /* alignment slack */ + stages * (PT + FT) * BK * 2 + staging_bufs * GROUP_BYTES + CTRL_BYTES;
 }
 
-// Chooses the N tile and the pipeline depth.  Eligible: dense, c_pad >= 8, im2col corner limits.
+// Chooses orientation, tiles and pipeline depth.  Eligible: dense, im2col corner limits.
 cprune_status plan_conv_tensor(cprune_plan *plan) {
     cprune_plan_info &i = plan->info;
     if (i.groups != 1) return CPRUNE_ERR_UNSUPPORTED;
     if (i.R > 16 || i.S > 16 || i.pad > 64 || i.stride > 8) return CPRUNE_ERR_UNSUPPORTED;
     if (i.W > 65535 || i.H > 65535) return CPRUNE_ERR_UNSUPPORTED;
     const long long M = (long long)i.N * i.P * i.Q;
-    const int tiles_m = (int)ceil_div(M, BM);
     const int k16 = round_up(i.K, 16);
-    // fewest N tiles that fit the 256-column accumulator, then split further while that fills
-    // more of the 148 SMs without dropping below 64 columns per tile
-    int tiles_n = (k16 + 255) / 256;
-    while (true) {
-        int next = tiles_n + 1;
-        int bn_next = round_up((k16 + next - 1) / next, 16);
-        if (bn_next < 64) break;
-        if ((long long)tiles_m * tiles_n >= 148) break;
-        tiles_n = next;
+    int PT, FT, tiles_n, bufs, group_rows;
+    if (i.K <= 128) {
+        // filters on the MMA-M side (padded to 128 rows), 256 pixels on the MMA-N side
+        plan->orient = ORIENT_FILT;
+        PT = 256; FT = 128; tiles_n = 1; bufs = 2; group_rows = 64;
+    } else {
+        plan->orient = ORIENT_PIX;
+        PT = 128; group_rows = 128; bufs = 2;
+        const int tiles_m = (int)ceil_div(M, PT);
+        // fewest filter tiles that fit the 256-column accumulator, then split further while that
+        // fills more of the 148 SMs without dropping below 128 filters per tile
+        tiles_n = (k16 + 255) / 256;
+        while (true) {
+            int next = tiles_n + 1;
+            int ft_next = round_up((k16 + next - 1) / next, 16);
+            if (ft_next < 128) break;
+            if ((long long)tiles_m * tiles_n >= 148) break;
+            tiles_n = next;
+        }
+        FT = round_up((k16 + tiles_n - 1) / tiles_n, 16);
+        tiles_n = (k16 + FT - 1) / FT;
     }
-    int BN = round_up((k16 + tiles_n - 1) / tiles_n, 16);
-    tiles_n = (k16 + BN - 1) / BN;
     int stages = MAX_STAGES;
-    while (stages > 2 && smem_for(stages, BN) > 200 * 1024) --stages;
-    i.tile_m = BM;
-    i.tile_n = BN;
+    while (stages > 2 && smem_for(stages, PT, FT, bufs, group_rows) > 227 * 1024) --stages;
+    i.tile_m = PT;
+    i.tile_n = FT;
     i.tile_k = BK;
     i.stages = stages;
-    i.tiles_m = tiles_m;
+    i.tiles_m = (int)ceil_div(M, PT);
     i.tiles_n = tiles_n;
-    i.k_alloc = tiles_n * BN;
+    i.k_alloc = tiles_n * FT;
     const int cblks = (i.c_pad + BK - 1) / BK;
     const int ksteps = (cblks - 1) * (BK / 16) + (i.c_pad - (cblks - 1) * BK + 15) / 16;
-    i.padded_flops = 2.0 * (double)tiles_m * BM * (double)i.k_alloc * (double)(i.R * i.S) * ksteps * 16.0;
-    plan->smem_bytes = smem_for(stages, BN);
+    i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * (double)(i.R * i.S) * ksteps * 16.0;
+    plan->staging_bufs = bufs;
+    plan->smem_bytes = smem_for(stages, PT, FT, bufs, group_rows);
     return CPRUNE_OK;
 }
 
-static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w) {
+static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w, void *y) {
     const cprune_plan_info &i = plan->info;
     cprune_status st = load_driver_entry_points();
     if (st != CPRUNE_OK) return st;
-    {
+    if (plan->map_x != x) {
         cuuint64_t dims[4] = {(cuuint64_t)i.c_pad, (cuuint64_t)i.W, (cuuint64_t)i.H, (cuuint64_t)i.N};
         cuuint64_t strides[3] = {(cuuint64_t)i.c_pad * 2, (cuuint64_t)i.W * i.c_pad * 2, (cuuint64_t)i.H * i.W * i.c_pad * 2};
         int lower[2] = {-i.pad, -i.pad};
         int upper[2] = {i.pad - (i.S - 1), i.pad - (i.R - 1)};
         cuuint32_t estr[4] = {1, (cuuint32_t)i.stride, (cuuint32_t)i.stride, 1};
         CUresult r = g_encode_im2col(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides,
-                                     lower, upper, BK, BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                     lower, upper, BK, (cuuint32_t)i.tile_m, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeIm2col");
         // Drivers up to 13.1 set a descriptor bit for im2col maps of tensors smaller than 128 KiB
         // that makes the load misbehave; the open-source CUTLASS im2col path clears it the same way.
         const size_t bytes = (size_t)i.N * i.H * i.W * i.c_pad * 2;
         if (g_driver_version <= 13010 && bytes < 131072) reinterpret_cast<uint64_t *>(&plan->tm_a)[1] &= ~(1ull << 21);
+        plan->map_x = x;
     }
-    {
+    if (plan->map_w != w) {
         cuuint64_t dims[3] = {(cuuint64_t)i.c_pad, (cuuint64_t)(i.R * i.S), (cuuint64_t)i.k_alloc};
         cuuint64_t strides[2] = {(cuuint64_t)i.c_pad * 2, (cuuint64_t)i.R * i.S * i.c_pad * 2};
         cuuint32_t box[3] = {BK, 1, (cuuint32_t)i.tile_n};
@@ -426,10 +605,22 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         CUresult r = g_encode_tiled(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box,
                                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(w)");
+        plan->map_w = w;
     }
-    plan->map_x = x;
-    plan->map_w = w;
+    if (plan->map_y != y) {
+        // output as a 2-D tensor [pixels][k_pad]; stored in boxes of 16 filters x 128 or 64 pixels
+        const long long M = (long long)i.N * i.P * i.Q;
+        cuuint64_t dims[2] = {(cuuint64_t)i.k_pad, (cuuint64_t)M};
+        cuuint64_t strides[1] = {(cuuint64_t)i.k_pad * 2};
+        cuuint32_t box[2] = {SUB, (cuuint32_t)(plan->orient == ORIENT_PIX ? 128 : 64)};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = g_encode_tiled(&plan->tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(y)");
+        plan->map_y = y;
+    }
     return CPRUNE_OK;
 }
 
@@ -446,22 +637,24 @@ static int sm_count() {
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
                                  void *y, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
-    CUtensorMap tm_a, tm_b;
+    CUtensorMap tm_x, tm_w, tm_y;
     {
         std::lock_guard<std::mutex> lock(plan->mu);
-        if (plan->map_x != x || plan->map_w != w) {
-            cprune_status s = encode_maps(plan, x, w);
+        if (plan->map_x != x || plan->map_w != w || plan->map_y != y) {
+            cprune_status s = encode_maps(plan, x, w, y);
             if (s != CPRUNE_OK) return s;
         }
-        std::memcpy(&tm_a, &plan->tm_a, sizeof(CUtensorMap));
-        std::memcpy(&tm_b, &plan->tm_b, sizeof(CUtensorMap));
+        std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
+        std::memcpy(&tm_w, &plan->tm_b, sizeof(CUtensorMap));
+        std::memcpy(&tm_y, &plan->tm_y, sizeof(CUtensorMap));
     }
     static std::mutex attr_mu;
     static int attr_set = 0;
     {
         std::lock_guard<std::mutex> lock(attr_mu);
         if (!attr_set) {
-            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_PIX>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_FILT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             attr_set = 1;
         }
     }
@@ -470,17 +663,20 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     p.P = i.P; p.Q = i.Q; p.stride = i.stride; p.pad = i.pad; p.R = i.R; p.S = i.S;
     p.cblks = (i.c_pad + BK - 1) / BK;
     p.ksteps_last = (i.c_pad - (p.cblks - 1) * BK + 15) / 16;
-    p.BN = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
+    p.PT = i.tile_m; p.FT = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
+    p.staging_bufs = plan->staging_bufs;
     p.act = plan->opts.activation;
     p.bias = b;
     p.res = (const __nv_bfloat16 *)res;
-    p.y = (__nv_bfloat16 *)y;
     p.status = device_status_word();
     if (!p.status) return cuda_fail(cudaGetLastError(), "status word");
     const int total = i.tiles_m * i.tiles_n;
     if (total == 0) return CPRUNE_OK;
     const int grid = total < sm_count() ? total : sm_count();
-    conv_tc_kernel<<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_a, tm_b, p);
+    if (plan->orient == ORIENT_PIX)
+        conv_tc_kernel<ORIENT_PIX><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, p);
+    else
+        conv_tc_kernel<ORIENT_FILT><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, p);
     CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
     return CPRUNE_OK;
 }

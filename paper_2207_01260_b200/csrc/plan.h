@@ -18,9 +18,13 @@ struct cprune_plan {
     std::mutex mu;
     const void *map_x = nullptr;
     const void *map_w = nullptr;
-    alignas(64) CUtensorMap tm_a;
-    alignas(64) CUtensorMap tm_b;
+    const void *map_y = nullptr;
+    alignas(64) CUtensorMap tm_a;   // activations (im2col mode)
+    alignas(64) CUtensorMap tm_b;   // packed filters
+    alignas(64) CUtensorMap tm_y;   // output, for the staged TMA stores
     int smem_bytes = 0;
+    int orient = 0;                 // which side of the MMA the pixels are on
+    int staging_bufs = 2;
 };
 
 namespace cprune {

@@ -39,8 +39,11 @@ def test_status_strings_and_padding(cp):
 def test_plan_shapes_and_families(cp):
     p = cp.cprune_task_plan(64, 64, 56, 56, 44, 3, 3, 1, 1)
     assert (p.P, p.Q, p.c_pad, p.k_pad) == (56, 56, 64, 48)
-    assert cp.KERNEL_NAMES[p.kernel] == "tensor" and p.tile_m == 128 and p.tile_n % 16 == 0
-    assert p.tiles_m == 64 * 56 * 56 // 128 and p.tiles_n * p.tile_n >= 44 and p.k_alloc == p.tiles_n * p.tile_n
+    # K <= 128: filters sit on the 128-row side of the MMA and a tile covers 256 pixels
+    assert cp.KERNEL_NAMES[p.kernel] == "tensor" and p.tile_m == 256 and p.tile_n == 128
+    assert p.tiles_m == 64 * 56 * 56 // 256 and p.tiles_n == 1 and p.k_alloc == 128
+    q = cp.cprune_task_plan(64, 256, 14, 14, 358, 3, 3, 1, 1)
+    assert q.tile_m == 128 and q.tile_n % 16 == 0 and q.tiles_n * q.tile_n >= 358 and q.k_alloc == q.tiles_n * q.tile_n
     assert p.flops == 2.0 * 64 * 44 * 64 * 56 * 56 * 9
     assert p.padded_flops >= p.flops
     p = cp.cprune_task_plan(1, 3, 224, 224, 64, 7, 7, 2, 3)
