@@ -52,7 +52,8 @@ struct TcParams {
     int ksteps_last;   // 16-channel MMA steps in the last channel block
     int PT, FT;        // pixels and filters per tile
     int tiles_m, tiles_n, k_pad, stages, act;
-    int staging_bufs;  // 1 or 2 staging buffers of PT_GROUP x 64 bf16
+    int small_c;       // c_pad == 8 (3-channel stems): a 64-wide K block is 8 taps x 8 channels
+    int iters;         // pipeline stages per tile (K blocks, plus residual blocks)
     const float *bias;
     const __nv_bfloat16 *res;
     int *status;
@@ -191,6 +192,18 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 
+// Descriptor of a K-major bf16 operand stored without swizzle as 8-row x 16-byte core matrices:
+// rows 16 bytes apart, 8-row groups 128 bytes apart, the next 8 channels `k_stride` bytes away
+// (the layout of one im2col TMA load of 8 channels per pixel; successive taps follow each other).
+__device__ __forceinline__ uint64_t smem_desc_interleaved(uint32_t addr, uint32_t k_stride) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((k_stride >> 4) & 0x3FFF) << 16;   // leading byte offset: next core matrix along K
+    d |= (uint64_t)(128 >> 4) << 32;                   // stride byte offset: next 8 rows
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+
 // Byte offset of (row, 16-byte half h) in a staged sub-tile of 32-byte rows under the 32-byte
 // swizzle (address bit 4 is XORed with bit 7, i.e. with bit 2 of the row).
 __device__ __forceinline__ uint32_t sub_off(int row, int h) { return (uint32_t)(row * 32 + ((h ^ ((row >> 2) & 1)) << 4)); }
@@ -213,7 +226,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     constexpr int GROUP_ROWS = ORIENT == ORIENT_PIX ? 128 : 64;
     constexpr int SUB_BYTES = GROUP_ROWS * SUB * 2;
     const uint32_t staging0 = base + (uint32_t)p.stages * stage_bytes;
-    const uint32_t ctrl0 = staging0 + (uint32_t)p.staging_bufs * GROUP_BYTES;
+    const uint32_t ctrl0 = staging0 + 2u * GROUP_BYTES;
     uint8_t *ctrl = smem + (ctrl0 - base);
     // barrier slots (8 bytes each): full[8], empty[8], tfull[2], tempty[2], epi[1]
     auto full_bar = [&](int s) { return ctrl0 + 8u * s; };
@@ -257,12 +270,38 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         uint32_t phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
+            const int mt = tile / p.tiles_n, nt_f = tile - mt * p.tiles_n;
             const long long m0 = (long long)mt * p.PT;
             const int n_img = (int)(m0 / PQ);
             const int rem = (int)(m0 - (long long)n_img * PQ);
             const int p0 = rem / p.Q, q0 = rem - p0 * p.Q;
             const int wc = q0 * p.stride - p.pad, hc = p0 * p.stride - p.pad;
+            if (p.small_c) {
+                // 8 taps x 8 channels per stage; every tap is its own im2col load of PT pixels x 16 bytes
+                const int taps = p.R * p.S;
+                for (int it = 0; it < p.iters; ++it) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                    if (!ok) break;
+                    if (elect_one()) {
+                        const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
+                        int nt = taps - it * 8;
+                        if (nt > 8) nt = 8;
+                        const int loads = (nt + 1) & ~1;      // an odd last tap is loaded twice: the MMA reads 2 taps
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(loads * p.PT * 16 + p.FT * BK * 2));
+                        for (int t = 0; t < loads; ++t) {
+                            int tap = it * 8 + t;
+                            if (tap >= taps) tap = taps - 1;  // finite filler; its weights are zero
+                            const int r = tap / p.S, s = tap - r * p.S;
+                            tma_load_im2col(x_dst + (uint32_t)(t * p.PT * 16), &tm_x, full_bar(stage), 0, wc, hc, n_img,
+                                            (uint16_t)s, (uint16_t)r);
+                        }
+                        tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), it * BK, 0, nt_f * p.FT);
+                    }
+                    __syncwarp();
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                continue;
+            }
             for (int r = 0; r < p.R && ok; ++r)
                 for (int s = 0; s < p.S && ok; ++s)
                     for (int cb = 0; cb < p.cblks; ++cb) {
@@ -272,7 +311,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                             const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
                             mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
                             tma_load_im2col(x_dst, &tm_x, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
-                            tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), cb * BK, r * p.S + s, nt * p.FT);
+                            tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), cb * BK, r * p.S + s, nt_f * p.FT);
                         }
                         __syncwarp();
                         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -292,15 +331,33 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_STRIDE);
             uint32_t accumulate = 0;
-            for (int tap = 0; tap < p.R * p.S && ok; ++tap)
-                for (int cb = 0; cb < p.cblks; ++cb) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag, p.status));
-                    if (!ok) break;
-                    const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
-                    const uint64_t dx = smem_desc_sw128(x_addr);
-                    const uint64_t dw = smem_desc_sw128(x_addr + x_bytes);
-                    const int nk = (cb == p.cblks - 1) ? p.ksteps_last : BK / 16;
-                    if (elect_one()) {
+            for (int it = 0; it < p.iters; ++it) {
+                ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag, p.status));
+                if (!ok) break;
+                const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
+                const uint64_t dw = smem_desc_sw128(x_addr + x_bytes);
+                int nk;
+                if (p.small_c) {
+                    int nt = p.R * p.S - it * 8;
+                    if (nt > 8) nt = 8;
+                    nk = (nt + 1) >> 1;
+                } else {
+                    nk = ((it + 1) % p.cblks == 0) ? p.ksteps_last : BK / 16;
+                }
+                if (elect_one()) {
+                    if (p.small_c) {
+                        // pixel operand: two taps (2 x 8 channels) per MMA, taps PT*16 bytes apart
+                        const uint32_t tap_bytes = (uint32_t)p.PT * 16u;
+                        for (int kk = 0; kk < nk; ++kk) {
+                            const uint64_t dxi = smem_desc_interleaved(x_addr + (uint32_t)(2 * kk) * tap_bytes, tap_bytes);
+                            if (ORIENT == ORIENT_PIX)
+                                umma_bf16(d_tmem, dxi, dw + (uint64_t)(2 * kk), idesc, accumulate);
+                            else
+                                umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dxi, idesc, accumulate);
+                            accumulate = 1;
+                        }
+                    } else {
+                        const uint64_t dx = smem_desc_sw128(x_addr);
                         for (int kk = 0; kk < nk; ++kk) {
                             // 16 channels = 32 bytes further along the swizzled row: +2 in 16-byte units
                             if (ORIENT == ORIENT_PIX)
@@ -309,12 +366,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                 umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dx + (uint64_t)(2 * kk), idesc, accumulate);
                             accumulate = 1;
                         }
-                        umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
                     }
-                    accumulate = 1;
-                    __syncwarp();
-                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
                 }
+                accumulate = 1;
+                __syncwarp();
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
             if (ok && elect_one()) umma_commit(tfull_bar(acc));
             __syncwarp();
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -538,6 +596,7 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     const long long M = (long long)i.N * i.P * i.Q;
     const int k16 = round_up(i.K, 16);
     int PT, FT, tiles_n, bufs, group_rows;
+    plan->small_c = (i.c_pad == 8 && i.K <= 128 && i.R * i.S > 1) ? 1 : 0;
     if (i.K <= 128) {
         // filters on the MMA-M side (padded to 128 rows), 256 pixels on the MMA-N side
         plan->orient = ORIENT_FILT;
@@ -571,6 +630,7 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     const int cblks = (i.c_pad + BK - 1) / BK;
     const int ksteps = (cblks - 1) * (BK / 16) + (i.c_pad - (cblks - 1) * BK + 15) / 16;
     i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * (double)(i.R * i.S) * ksteps * 16.0;
+    if (plan->small_c) i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * ((i.R * i.S + 1) / 2) * 16.0;
     plan->staging_bufs = bufs;
     plan->smem_bytes = smem_for(stages, PT, FT, bufs, group_rows);
     return CPRUNE_OK;
@@ -586,10 +646,12 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         int lower[2] = {-i.pad, -i.pad};
         int upper[2] = {i.pad - (i.S - 1), i.pad - (i.R - 1)};
         cuuint32_t estr[4] = {1, (cuuint32_t)i.stride, (cuuint32_t)i.stride, 1};
+        // small-C mode: 8 channels (16 bytes) per pixel, dense rows, no swizzle
         CUresult r = g_encode_im2col(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides,
-                                     lower, upper, BK, (cuuint32_t)i.tile_m, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                     lower, upper, plan->small_c ? 8 : BK, (cuuint32_t)i.tile_m, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                     plan->small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeIm2col");
         // Drivers up to 13.1 set a descriptor bit for im2col maps of tensors smaller than 128 KiB
         // that makes the load misbehave; the open-source CUTLASS im2col path clears it the same way.
@@ -598,8 +660,10 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         plan->map_x = x;
     }
     if (plan->map_w != w) {
-        cuuint64_t dims[3] = {(cuuint64_t)i.c_pad, (cuuint64_t)(i.R * i.S), (cuuint64_t)i.k_alloc};
-        cuuint64_t strides[2] = {(cuuint64_t)i.c_pad * 2, (cuuint64_t)i.R * i.S * i.c_pad * 2};
+        // small-C mode reads a filter row [R*S taps][8 channels] as one long channel axis
+        cuuint64_t dims[3] = {(cuuint64_t)(plan->small_c ? i.R * i.S * 8 : i.c_pad), (cuuint64_t)(plan->small_c ? 1 : i.R * i.S),
+                              (cuuint64_t)i.k_alloc};
+        cuuint64_t strides[2] = {(cuuint64_t)(plan->small_c ? i.R * i.S * 8 : i.c_pad) * 2, (cuuint64_t)i.R * i.S * i.c_pad * 2};
         cuuint32_t box[3] = {BK, 1, (cuuint32_t)i.tile_n};
         cuuint32_t estr[3] = {1, 1, 1};
         CUresult r = g_encode_tiled(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box,
@@ -664,7 +728,8 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     p.cblks = (i.c_pad + BK - 1) / BK;
     p.ksteps_last = (i.c_pad - (p.cblks - 1) * BK + 15) / 16;
     p.PT = i.tile_m; p.FT = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
-    p.staging_bufs = plan->staging_bufs;
+    p.small_c = plan->small_c;
+    p.iters = plan->small_c ? (i.R * i.S + 7) / 8 : i.R * i.S * p.cblks;
     p.act = plan->opts.activation;
     p.bias = b;
     p.res = (const __nv_bfloat16 *)res;

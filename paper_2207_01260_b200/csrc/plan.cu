@@ -51,7 +51,8 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
         i.tile_k = 8;
     } else {
         if (family == CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;
-        if (family == CPRUNE_KERNEL_AUTO) family = i.C < 8 ? CPRUNE_KERNEL_DIRECT : CPRUNE_KERNEL_TENSOR;
+        // 3-channel stems run on the tensor cores too when their filters fit the 128-row side
+        if (family == CPRUNE_KERNEL_AUTO) family = (i.C < 8 && i.K > 128) ? CPRUNE_KERNEL_DIRECT : CPRUNE_KERNEL_TENSOR;
         if (st == CPRUNE_OK && family == CPRUNE_KERNEL_TENSOR) {
             cprune_status t = plan_conv_tensor(pl);
             if (t != CPRUNE_OK) {

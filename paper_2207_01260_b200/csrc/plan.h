@@ -25,6 +25,7 @@ struct cprune_plan {
     int smem_bytes = 0;
     int orient = 0;                 // which side of the MMA the pixels are on
     int staging_bufs = 2;
+    int small_c = 0;                // 3-channel stems: 8 taps x 8 channels per K block
 };
 
 namespace cprune {

@@ -163,11 +163,16 @@ def test_every_channel_residue(cp, C):
     check_task(cp, 1, C, 10, 10, C + 3, 3, 1, 1, kernel="tensor")
 
 
-def test_small_stem_shapes_use_the_direct_kernel(cp):
-    plan = check_task(cp, 1, 3, 32, 32, 45, 3, 1, 1)
-    assert cp.KERNEL_NAMES[plan.kernel] == "direct"
-    check_task(cp, 1, 3, 37, 37, 64, 7, 2, 3)
-    check_task(cp, 2, 3, 30, 30, 32, 3, 2, 1, act="relu6")
+@pytest.mark.parametrize("kernel", ["tensor", "direct"])
+def test_three_channel_stems(cp, kernel):
+    # 3 input channels: the tensor-core kernel packs 8 taps x 8 padded channels into one K block
+    plan = check_task(cp, 1, 3, 32, 32, 45, 3, 1, 1, kernel=kernel)
+    assert cp.KERNEL_NAMES[plan.kernel] == kernel
+    check_task(cp, 1, 3, 37, 37, 64, 7, 2, 3, kernel=kernel)
+    check_task(cp, 2, 3, 30, 30, 32, 3, 2, 1, act="relu6", kernel=kernel)
+    check_task(cp, 3, 3, 64, 64, 64, 7, 2, 3, kernel=kernel)
+    check_task(cp, 2, 5, 21, 19, 24, 5, 1, 2, kernel=kernel)
+    assert cp.KERNEL_NAMES[cp.cprune_task_plan(1, 3, 224, 224, 64, 7, 7, 2, 3).kernel] == "tensor"
 
 
 @pytest.mark.parametrize("C,H,W,stride", [(32, 16, 16, 1), (72, 15, 17, 2), (108, 14, 14, 1), (144, 7, 9, 2),
@@ -291,13 +296,13 @@ def test_vgg16_cifar_parity(cp):
 def test_resnet18_parity(cp):
     net, _, _ = model_parity(cp, "resnet18", 2)
     kinds = {cp.KERNEL_NAMES[i["kernel"]] for i in net.conv_launch_info().values()}
-    assert kinds == {"tensor", "direct"}                # the 3-channel stem is the only direct task
+    assert kinds == {"tensor"}
 
 
 def test_mobilenet_v2_parity(cp):
     net, _, _ = model_parity(cp, "mobilenet_v2", 2)
     kinds = {cp.KERNEL_NAMES[i["kernel"]] for i in net.conv_launch_info().values()}
-    assert kinds == {"tensor", "direct", "depthwise"}
+    assert kinds == {"tensor", "depthwise"}
 
 
 def test_intermediate_activations_match(cp):

@@ -47,7 +47,9 @@ def test_plan_shapes_and_families(cp):
     assert p.flops == 2.0 * 64 * 44 * 64 * 56 * 56 * 9
     assert p.padded_flops >= p.flops
     p = cp.cprune_task_plan(1, 3, 224, 224, 64, 7, 7, 2, 3)
-    assert (p.P, p.Q) == (112, 112) and cp.KERNEL_NAMES[p.kernel] == "direct"
+    assert (p.P, p.Q) == (112, 112) and cp.KERNEL_NAMES[p.kernel] == "tensor"
+    p = cp.cprune_task_plan(1, 3, 224, 224, 64, 7, 7, 2, 3, kernel="direct")
+    assert cp.KERNEL_NAMES[p.kernel] == "direct"
     p = cp.cprune_task_plan(8, 108, 56, 56, 108, 3, 3, 2, 1, groups=108, activation="relu6")
     assert cp.KERNEL_NAMES[p.kernel] == "depthwise" and (p.P, p.Q) == (28, 28) and p.c_pad == 112
     assert p.flops == 2.0 * 8 * 108 * 28 * 28 * 9
