@@ -54,6 +54,7 @@ struct TcParams {
     int tiles_m, tiles_n, k_pad, stages, act;
     int small_c;       // c_pad == 8 (3-channel stems): a 64-wide K block is 8 taps x 8 channels
     int iters;         // pipeline stages per tile (K blocks, plus residual blocks)
+    int res_iters;     // ORIENT_FILT with a residual: trailing stages that add it on the tensor core
     const float *bias;
     const __nv_bfloat16 *res;
     int *status;
@@ -127,6 +128,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         " [%0], [%1, {%3, %4, %5}], [%2];"
         :
         : "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];"
+        :
+        : "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
         : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
@@ -213,7 +222,8 @@ __device__ __forceinline__ uint32_t sub_off(int row, int h) { return (uint32_t)(
 template <int ORIENT>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-               const __grid_constant__ CUtensorMap tm_y, const TcParams p) {
+               const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res,
+               const __grid_constant__ CUtensorMap tm_id, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
@@ -279,7 +289,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             if (p.small_c) {
                 // 8 taps x 8 channels per stage; every tap is its own im2col load of PT pixels x 16 bytes
                 const int taps = p.R * p.S;
-                for (int it = 0; it < p.iters; ++it) {
+                for (int it = 0; it < p.iters - p.res_iters; ++it) {
                     ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                     if (!ok) break;
                     if (elect_one()) {
@@ -300,8 +310,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
-                continue;
-            }
+            } else {
             for (int r = 0; r < p.R && ok; ++r)
                 for (int s = 0; s < p.S && ok; ++s)
                     for (int cb = 0; cb < p.cblks; ++cb) {
@@ -316,6 +325,22 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                         __syncwarp();
                         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                     }
+            }
+            // residual blocks (ORIENT_FILT): the residual tile [PT pixels][64 filters] is the pixel-side
+            // operand and a 64-column slice of the identity matrix the filter-side operand, so that the
+            // MMA adds residual[pixel][k] to accumulator row k
+            for (int j = 0; j < p.res_iters && ok; ++j) {
+                ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
+                    mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
+                    tma_load_2d(x_dst, &tm_res, full_bar(stage), j * BK, (int)m0);
+                    tma_load_2d(x_dst + x_bytes, &tm_id, full_bar(stage), j * BK, 0);
+                }
+                __syncwarp();
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issue
@@ -337,7 +362,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
                 const uint64_t dw = smem_desc_sw128(x_addr + x_bytes);
                 int nk;
-                if (p.small_c) {
+                const int main_iters = p.iters - p.res_iters;
+                const bool res_it = it >= main_iters;
+                if (res_it) {
+                    int left = p.k_pad - (it - main_iters) * BK;
+                    if (left > BK) left = BK;
+                    nk = (left + 15) >> 4;
+                } else if (p.small_c) {
                     int nt = p.R * p.S - it * 8;
                     if (nt > 8) nt = 8;
                     nk = (nt + 1) >> 1;
@@ -345,7 +376,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     nk = ((it + 1) % p.cblks == 0) ? p.ksteps_last : BK / 16;
                 }
                 if (elect_one()) {
-                    if (p.small_c) {
+                    if (p.small_c && !res_it) {
                         // pixel operand: two taps (2 x 8 channels) per MMA, taps PT*16 bytes apart
                         const uint32_t tap_bytes = (uint32_t)p.PT * 16u;
                         for (int kk = 0; kk < nk; ++kk) {
@@ -491,15 +522,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     if (warp_has_work) {
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
-                            // residual values of 32 pixels for this filter, all loads in flight together
-                            unsigned short rr[32];
-                            const bool has_res = p.res != nullptr && k_ok;
-                            if (has_res) {
-                                const unsigned short *rp = (const unsigned short *)p.res + (size_t)(mg + half * 32) * p.k_pad + k;
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    rr[j] = (mg + half * 32 + j < p.M) ? __ldg(rp + (size_t)j * p.k_pad) : (unsigned short)0;
-                            }
                             uint32_t v[32];
                             tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32), v);
                             tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32 + 16), v + 16);
@@ -509,7 +531,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                 for (int j = 0; j < 32; ++j) {
                                     const int px = half * 32 + j;
                                     float f = __uint_as_float(v[j]) + bias;
-                                    if (has_res) f += __uint_as_float((uint32_t)rr[j] << 16);
                                     f = apply_act(f, p.act);
                                     *(__nv_bfloat16 *)(dst + sub_off(px, hk)) = __float2bfloat16_rn(f);
                                 }
@@ -582,6 +603,35 @@ static cprune_status load_driver_entry_points() {
     return CPRUNE_OK;
 }
 
+// 128 x 128 identity in bf16: the filter-side operand of the residual blocks (see the producer).
+static __device__ __align__(256) __nv_bfloat16 g_identity[128 * 128];
+
+__global__ void fill_identity_kernel() {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < 128 * 128) g_identity[i] = __float2bfloat16_rn((i / 128 == i % 128) ? 1.f : 0.f);
+}
+
+// Device address of the identity matrix on the current device; filled on first use (one small
+// launch on the given stream, ordered before the conv kernel that follows it there).
+static cprune_status identity_address(void **out, cudaStream_t st) {
+    static std::mutex mu;
+    static void *ptrs[64] = {nullptr};
+    int dev = 0;
+    CPRUNE_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CPRUNE_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void *p = nullptr;
+        CPRUNE_CUDA_CHECK(cudaGetSymbolAddress(&p, g_identity));
+        fill_identity_kernel<<<64, 256, 0, st>>>();
+        CPRUNE_LAUNCH_CHECK("fill_identity_kernel");
+        CPRUNE_CUDA_CHECK(cudaStreamSynchronize(st));   // later launches may come from other streams
+        ptrs[dev] = p;
+    }
+    *out = ptrs[dev];
+    return CPRUNE_OK;
+}
+
 static int smem_for(int stages, int PT, int FT, int staging_bufs, int group_rows) {
     (void)group_rows;
     return 1024 /* alignment slack */ + stages * (PT + FT) * BK * 2 + staging_bufs * GROUP_BYTES + CTRL_BYTES;
@@ -636,7 +686,8 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     return CPRUNE_OK;
 }
 
-static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w, void *y) {
+static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w, void *y, const void *res,
+                                 cudaStream_t stream) {
     const cprune_plan_info &i = plan->info;
     cprune_status st = load_driver_entry_points();
     if (st != CPRUNE_OK) return st;
@@ -685,6 +736,29 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(y)");
         plan->map_y = y;
     }
+    if (plan->orient == ORIENT_FILT && res && plan->map_res != res) {
+        // residual [pixels][k_pad], loaded as the pixel-side operand: 64 filters x 256 pixels
+        const long long M = (long long)i.N * i.P * i.Q;
+        cuuint64_t dims[2] = {(cuuint64_t)i.k_pad, (cuuint64_t)M};
+        cuuint64_t strides[1] = {(cuuint64_t)i.k_pad * 2};
+        cuuint32_t box[2] = {BK, (cuuint32_t)i.tile_m};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = g_encode_tiled(&plan->tm_res, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(res), dims, strides,
+                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(res)");
+        void *ident = nullptr;
+        cprune_status s2 = identity_address(&ident, stream);
+        if (s2 != CPRUNE_OK) return s2;
+        cuuint64_t idims[2] = {128, 128};
+        cuuint64_t istrides[1] = {256};
+        cuuint32_t ibox[2] = {BK, 128};
+        r = g_encode_tiled(&plan->tm_id, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ident, idims, istrides, ibox, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(identity)");
+        plan->map_res = res;
+    }
     return CPRUNE_OK;
 }
 
@@ -701,16 +775,20 @@ static int sm_count() {
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
                                  void *y, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
-    CUtensorMap tm_x, tm_w, tm_y;
+    CUtensorMap tm_x, tm_w, tm_y, tm_res, tm_id;
+    const bool mma_res = plan->orient == ORIENT_FILT && res != nullptr;
     {
         std::lock_guard<std::mutex> lock(plan->mu);
-        if (plan->map_x != x || plan->map_w != w || plan->map_y != y) {
-            cprune_status s = encode_maps(plan, x, w, y);
+        if (plan->map_x != x || plan->map_w != w || plan->map_y != y || (mma_res && plan->map_res != res)) {
+            cprune_status s = encode_maps(plan, x, w, y, res, st);
             if (s != CPRUNE_OK) return s;
         }
         std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
         std::memcpy(&tm_w, &plan->tm_b, sizeof(CUtensorMap));
         std::memcpy(&tm_y, &plan->tm_y, sizeof(CUtensorMap));
+        // without a tensor-core residual the two extra maps are never read; pass valid copies anyway
+        std::memcpy(&tm_res, mma_res ? &plan->tm_res : &plan->tm_y, sizeof(CUtensorMap));
+        std::memcpy(&tm_id, mma_res ? &plan->tm_id : &plan->tm_y, sizeof(CUtensorMap));
     }
     static std::mutex attr_mu;
     static int attr_set = 0;
@@ -729,19 +807,20 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     p.ksteps_last = (i.c_pad - (p.cblks - 1) * BK + 15) / 16;
     p.PT = i.tile_m; p.FT = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
     p.small_c = plan->small_c;
-    p.iters = plan->small_c ? (i.R * i.S + 7) / 8 : i.R * i.S * p.cblks;
+    p.res_iters = mma_res ? (i.k_pad + BK - 1) / BK : 0;
+    p.iters = (plan->small_c ? (i.R * i.S + 7) / 8 : i.R * i.S * p.cblks) + p.res_iters;
     p.act = plan->opts.activation;
     p.bias = b;
-    p.res = (const __nv_bfloat16 *)res;
+    p.res = mma_res ? nullptr : (const __nv_bfloat16 *)res;   // ORIENT_PIX adds it in the epilogue
     p.status = device_status_word();
     if (!p.status) return cuda_fail(cudaGetLastError(), "status word");
     const int total = i.tiles_m * i.tiles_n;
     if (total == 0) return CPRUNE_OK;
     const int grid = total < sm_count() ? total : sm_count();
     if (plan->orient == ORIENT_PIX)
-        conv_tc_kernel<ORIENT_PIX><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, p);
+        conv_tc_kernel<ORIENT_PIX><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
     else
-        conv_tc_kernel<ORIENT_FILT><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, p);
+        conv_tc_kernel<ORIENT_FILT><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
     CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
     return CPRUNE_OK;
 }

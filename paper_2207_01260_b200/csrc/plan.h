@@ -19,9 +19,12 @@ struct cprune_plan {
     const void *map_x = nullptr;
     const void *map_w = nullptr;
     const void *map_y = nullptr;
+    const void *map_res = nullptr;
     alignas(64) CUtensorMap tm_a;   // activations (im2col mode)
     alignas(64) CUtensorMap tm_b;   // packed filters
     alignas(64) CUtensorMap tm_y;   // output, for the staged TMA stores
+    alignas(64) CUtensorMap tm_res; // residual as an MMA operand (filter-major orientation)
+    alignas(64) CUtensorMap tm_id;  // identity matrix
     int smem_bytes = 0;
     int orient = 0;                 // which side of the MMA the pixels are on
     int staging_bufs = 2;

@@ -57,44 +57,46 @@ __global__ void __launch_bounds__(128) gap_kernel(const bf16x8 *__restrict__ x, 
     y[e] = pack8(s);
 }
 
-// one warp per output feature o, looping over the images of the batch in groups of NB so that a
-// weight row is read once per group
+// one warp per (output feature o, group of NB images): the warp reads the weight row once and
+// NB activation rows, reduces with shuffles; warps of a block share o when there are enough groups,
+// so the weight row is fetched from L2 once per block
 template <int NB>
 __global__ void __launch_bounds__(256) fc_kernel(const bf16x8 *__restrict__ x, int N, int in8,
                                                  const bf16x8 *__restrict__ w, const float *__restrict__ b, int out,
                                                  int out_pad, int act, int out_is_f32, void *__restrict__ y) {
-    int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    int lane = threadIdx.x & 31;
-    if (o >= out_pad) return;
+    const int ngroups = (N + NB - 1) / NB;
+    const long long widx = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (widx >= (long long)out_pad * ngroups) return;
+    const int o = (int)(widx / ngroups);
+    const int n0 = (int)(widx - (long long)o * ngroups) * NB;
     const bf16x8 *wr = w + (size_t)o * in8;
-    for (int n0 = 0; n0 < N; n0 += NB) {
-        float acc[NB];
+    float acc[NB];
 #pragma unroll
-        for (int j = 0; j < NB; ++j) acc[j] = 0.f;
-        for (int i = lane; i < in8; i += 32) {
-            float wf[8];
-            unpack8(ldg8(wr + i), wf);
-#pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                if (n0 + j < N) {
-                    float xf[8];
-                    unpack8(ldg8(x + (size_t)(n0 + j) * in8 + i), xf);
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) acc[j] = fmaf(xf[t], wf[t], acc[j]);
-                }
-            }
-        }
+    for (int j = 0; j < NB; ++j) acc[j] = 0.f;
+    for (int i = lane; i < in8; i += 32) {
+        float wf[8];
+        unpack8(ldg8(wr + i), wf);
 #pragma unroll
         for (int j = 0; j < NB; ++j) {
-            float v = acc[j];
-            for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-            if (lane == 0 && n0 + j < N) {
-                v = apply_act(v + b[o], act);
-                if (out_is_f32) {
-                    if (o < out) ((float *)y)[(size_t)(n0 + j) * out + o] = v;
-                } else {
-                    ((__nv_bfloat16 *)y)[(size_t)(n0 + j) * out_pad + o] = __float2bfloat16_rn(o < out ? v : 0.f);
-                }
+            if (n0 + j < N) {
+                float xf[8];
+                unpack8(ldg8(x + (size_t)(n0 + j) * in8 + i), xf);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[j] = fmaf(xf[t], wf[t], acc[j]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < NB; ++j) {
+        float v = acc[j];
+        for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+        if (lane == 0 && n0 + j < N) {
+            v = apply_act(v + b[o], act);
+            if (out_is_f32) {
+                if (o < out) ((float *)y)[(size_t)(n0 + j) * out + o] = v;
+            } else {
+                ((__nv_bfloat16 *)y)[(size_t)(n0 + j) * out_pad + o] = __float2bfloat16_rn(o < out ? v : 0.f);
             }
         }
     }
@@ -139,8 +141,9 @@ cprune_status cprune_fc(const void *x, int N, int in, const void *w_packed, cons
                         int out_is_f32, void *y, void *stream) {
     if (!x || !w_packed || !b_packed || !y || N <= 0 || in <= 0 || out <= 0) return CPRUNE_ERR_INVALID_ARG;
     int in8 = cprune_padded_channels(in) / 8, out_pad = cprune_padded_channels(out);
-    int warps = 8;
-    fc_kernel<8><<<(out_pad + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(
+    const int warps = 8;
+    const long long total_warps = (long long)out_pad * ((N + 7) / 8);
+    fc_kernel<8><<<(unsigned)((total_warps + warps - 1) / warps), warps * 32, 0, (cudaStream_t)stream>>>(
         (const bf16x8 *)x, N, in8, (const bf16x8 *)w_packed, b_packed, out, out_pad, act, out_is_f32, y);
     CPRUNE_LAUNCH_CHECK("fc_kernel");
     return CPRUNE_OK;
