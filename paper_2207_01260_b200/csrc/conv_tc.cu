@@ -632,6 +632,22 @@ static cprune_status identity_address(void **out, cudaStream_t st) {
     return CPRUNE_OK;
 }
 
+// Tiled bf16 tensor map without swizzle (used by the depthwise kernel for its input patches).
+cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
+                                const unsigned long long *strides_bytes, const unsigned *box) {
+    cprune_status st = load_driver_entry_points();
+    if (st != CPRUNE_OK) return st;
+    cuuint64_t d[5], s[4];
+    cuuint32_t b[5], e[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; e[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
+    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(ptr), d, s, b, e,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(depthwise)");
+    return CPRUNE_OK;
+}
+
 static int smem_for(int stages, int PT, int FT, int staging_bufs, int group_rows) {
     (void)group_rows;
     return 1024 /* alignment slack */ + stages * (PT + FT) * BK * 2 + staging_bufs * GROUP_BYTES + CTRL_BYTES;

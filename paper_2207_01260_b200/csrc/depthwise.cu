@@ -1,112 +1,231 @@
 // Depthwise 3x3 task (groups == C == K): memory-bound, CUDA cores.  bf16 NHWC in and out with
-// padded channels, float32 arithmetic, fused bias + activation (+ residual).  Threads are laid out
-// with the channel group fastest, so that a warp reads consecutive 16-byte vectors of one pixel
-// and its neighbours; each thread produces TQ adjacent output columns and reuses the input
-// columns they share.
+// padded channels, float32 arithmetic, fused bias + activation (+ residual).
+//
+// One CTA computes TH x TW output pixels of one image for one block of 64 channels.  Its input
+// patch ((TH-1)*stride+3) x ((TW-1)*stride+3) pixels x 64 channels comes in with a single tiled
+// TMA load (out-of-bounds pixels and channels read as zero, which is the padding), so every input
+// byte is fetched from L2/HBM once per CTA and the nine taps are served from shared memory.
+// A thread owns 8 channels of one output column and walks down the TH rows; threads of a warp
+// cover the 8 channel groups of 4 neighbouring columns, i.e. four contiguous 128-byte pixels.
+// Several CTAs share an SM, so one CTA's load overlaps the arithmetic of the others.  The wait
+// on the load is bounded like every other device-side wait of the library.
+#include <cstring>
+
 #include "common.cuh"
 #include "plan.h"
 
 namespace cprune {
 
 struct DwParams {
-    const bf16x8 *x;
     const bf16x8 *w;   // [3][3][c8]
     const float *b;
     const bf16x8 *res;
     bf16x8 *y;
-    int N, H, W, P, Q, stride, pad, act;
-    int c8;
-    int qt;            // ceil(Q / TQ)
-    long long items;   // N * P * qt * c8
+    int P, Q, pad, act;
+    int c8;            // c_pad / 8
+    int G;             // channel groups (of 8) per CTA: min(8, c8)
+    int TH, TW, IH, IW;
+    int tiles_h, tiles_w, cblocks;
+    int *status;
 };
 
-template <int TQ, int STRIDE>
-__global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p) {
-    long long item = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (item >= p.items) return;
-    int cg = (int)(item % p.c8);
-    long long t = item / p.c8;
-    int qb = (int)(t % p.qt) * TQ;
-    t /= p.qt;
-    int pp = (int)(t % p.P);
-    int n = (int)(t / p.P);
+__device__ __forceinline__ uint32_t dw_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-    constexpr int COLS = (TQ - 1) * STRIDE + 3;  // input columns feeding TQ outputs
-    float acc[TQ][8];
-#pragma unroll
-    for (int j = 0; j < TQ; ++j)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[j][i] = 0.f;
+template <int STRIDE>
+__global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant__ CUtensorMap tm_x, const DwParams p) {
+    extern __shared__ __align__(128) uint8_t dw_smem[];
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int failed;
 
-    const int v0 = qb * STRIDE - p.pad;
+    int bid = blockIdx.x;
+    const int cb = bid % p.cblocks; bid /= p.cblocks;
+    const int tw = bid % p.tiles_w; bid /= p.tiles_w;
+    const int th = bid % p.tiles_h;
+    const int n = bid / p.tiles_h;
+    const int p0 = th * p.TH, q0 = tw * p.TW;
+    const int G = p.G;
+
+    const uint32_t bar_a = dw_smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        failed = 0;
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const uint32_t bytes = (uint32_t)(p.IH * p.IW * G * 16);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(bytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+            :
+            : "r"(dw_smem_u32(dw_smem)), "l"(&tm_x), "r"(bar_a), "r"(cb * G * 8), "r"(q0 * STRIDE - p.pad),
+              "r"(p0 * STRIDE - p.pad), "r"(n)
+            : "memory");
+    }
+    __syncthreads();   // the barrier is initialised before anyone polls it
+
+    const int cg = threadIdx.x % G;          // channel group within the CTA's channel block
+    const int qq = threadIdx.x / G;          // output column within the tile
+    const int cgg = cb * G + cg;             // channel group within the tensor
+    const bool active = qq < p.TW && q0 + qq < p.Q && cgg < p.c8;
+
+    // filter taps (float32) and bias of this thread's 8 channels (overlaps the load)
+    float wf[9][8];
+    float bf[8];
+    if (active) {
 #pragma unroll
-    for (int r = 0; r < 3; ++r) {
-        int h = pp * STRIDE - p.pad + r;
-        if (h < 0 || h >= p.H) continue;
-        float wf[3][8];
+        for (int t = 0; t < 9; ++t) unpack8(ldg8(p.w + (size_t)t * p.c8 + cgg), wf[t]);
 #pragma unroll
-        for (int s = 0; s < 3; ++s) unpack8(ldg8(p.w + (size_t)(r * 3 + s) * p.c8 + cg), wf[s]);
-        const bf16x8 *row = p.x + ((size_t)n * p.H + h) * p.W * p.c8 + cg;
-#pragma unroll
-        for (int col = 0; col < COLS; ++col) {
-            int v = v0 + col;
-            if (v < 0 || v >= p.W) continue;
-            float xf[8];
-            unpack8(ldg8(row + (size_t)v * p.c8), xf);
-#pragma unroll
-            for (int j = 0; j < TQ; ++j) {
-                int s = col - j * STRIDE;
-                if (s >= 0 && s < 3) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(xf[i], wf[s][i], acc[j][i]);
-                }
+        for (int i = 0; i < 8; ++i) bf[i] = __ldg(p.b + cgg * 8 + i);
+    }
+
+    // bounded wait for the patch
+    {
+        uint32_t ok = 0;
+        long long t0 = clock64();
+        while (true) {
+            asm volatile(
+                "{\n\t.reg .pred q;\n\t"
+                "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\n\t"
+                "selp.u32 %0, 1, 0, q;\n\t}"
+                : "=r"(ok)
+                : "r"(bar_a)
+                : "memory");
+            if (ok) break;
+            if (clock64() - t0 > (1LL << 31)) {
+                atomicOr(p.status, STATUS_TIMEOUT);
+                failed = 1;
+                break;
             }
         }
     }
-    float bf[8];
+    __syncthreads();
+    if (failed) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let a late copy land before the CTA's memory goes away
+        return;
+    }
+    if (!active) return;
+
+    const bf16x8 *patch = reinterpret_cast<const bf16x8 *>(dw_smem) + cg;   // [IH][IW][G groups]
+    const size_t out_row = (size_t)p.Q * p.c8;
+    const size_t o0 = (((size_t)n * p.P + p0) * p.Q + q0 + qq) * p.c8 + cgg;
+
+    auto finish = [&](float *acc, int pp) {
+        const size_t o = o0 + (size_t)pp * out_row;
+        if (p.res) {
+            float rf[8];
+            unpack8(ldg8(p.res + o), rf);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) bf[i] = p.b[cg * 8 + i];
-#pragma unroll
-    for (int j = 0; j < TQ; ++j) {
-        int q = qb + j;
-        if (q >= p.Q) break;
-        size_t o = (((size_t)n * p.P + pp) * p.Q + q) * p.c8 + cg;
-        float rf[8];
-        if (p.res) unpack8(p.res[o], rf);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float v = acc[j][i] + bf[i];
-            if (p.res) v += rf[i];
-            acc[j][i] = apply_act(v, p.act);
+            for (int i = 0; i < 8; ++i) acc[i] += rf[i];
         }
-        p.y[o] = pack8(acc[j]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = apply_act(acc[i], p.act);
+        p.y[o] = pack8(acc);
+    };
+
+    if (STRIDE == 1) {
+        // walk down the input rows; each row feeds the three output rows it overlaps
+        const int rows = min(p.TH, p.P - p0);       // output rows of this tile
+        float a0[8], a1[8], a2[8];                  // accumulators of output rows h-2, h-1, h
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { a0[i] = bf[i]; a1[i] = bf[i]; a2[i] = bf[i]; }
+        for (int h = 0; h < rows + 2; ++h) {
+            const bf16x8 *row = patch + ((size_t)h * p.IW + qq) * G;
+            float x[3][8];
+#pragma unroll
+            for (int s = 0; s < 3; ++s) unpack8(row[s * G], x[s]);
+#pragma unroll
+            for (int s = 0; s < 3; ++s)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    a0[i] = fmaf(x[s][i], wf[6 + s][i], a0[i]);   // this row is tap row 2 of output row h-2
+                    a1[i] = fmaf(x[s][i], wf[3 + s][i], a1[i]);   // tap row 1 of output row h-1
+                    a2[i] = fmaf(x[s][i], wf[s][i], a2[i]);       // tap row 0 of output row h
+                }
+            if (h >= 2) finish(a0, h - 2);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { a0[i] = a1[i]; a1[i] = a2[i]; a2[i] = bf[i]; }
+        }
+    } else {
+        for (int pp = 0; pp < p.TH && p0 + pp < p.P; ++pp) {
+            float acc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = bf[i];
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                const bf16x8 *row = patch + ((size_t)(pp * STRIDE + r) * p.IW + qq * STRIDE) * G;
+#pragma unroll
+                for (int s = 0; s < 3; ++s) {
+                    float xf[8];
+                    unpack8(row[s * G], xf);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(xf[i], wf[r * 3 + s][i], acc[i]);
+                }
+            }
+            finish(acc, pp);
+        }
     }
 }
 
-cprune_status launch_depthwise(const cprune_plan *plan, const void *x, const void *w, const float *b,
-                               const void *res, void *y, cudaStream_t st) {
+// Tile of output pixels per CTA and channel groups per CTA.
+static void dw_tile(const cprune_plan_info &i, int *TH, int *TW, int *G) {
+    const int c8 = i.c_pad / 8;
+    *G = c8 < 8 ? c8 : 8;
+    int tw = 224 / *G;                      // about 224 threads per CTA
+    if (i.stride == 2 && tw > 28) tw = 28;  // keeps the input patch small
+    *TW = i.Q < tw ? i.Q : tw;
+    int th = i.stride == 1 ? 14 : (*TW <= 14 ? 7 : 4);
+    *TH = i.P < th ? i.P : th;
+}
+
+cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
+                               void *y, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
     DwParams p;
-    p.x = (const bf16x8 *)x;
     p.w = (const bf16x8 *)w;
     p.b = b;
     p.res = (const bf16x8 *)res;
     p.y = (bf16x8 *)y;
-    p.N = i.N; p.H = i.H; p.W = i.W; p.P = i.P; p.Q = i.Q;
-    p.stride = i.stride; p.pad = i.pad; p.act = plan->opts.activation;
+    p.P = i.P; p.Q = i.Q; p.pad = i.pad; p.act = plan->opts.activation;
     p.c8 = i.c_pad / 8;
-    const int TQ = i.tile_n;  // output columns per thread, chosen by the plan
-    p.qt = (i.Q + TQ - 1) / TQ;
-    p.items = (long long)i.N * i.P * p.qt * p.c8;
-    if (p.items == 0) return CPRUNE_OK;
-    long long blocks = ceil_div(p.items, 256);
-    if (blocks > 0x7fffffffLL) return CPRUNE_ERR_UNSUPPORTED;
-    if (i.stride == 1 && TQ == 4) depthwise3x3_kernel<4, 1><<<(unsigned)blocks, 256, 0, st>>>(p);
-    else if (i.stride == 1 && TQ == 2) depthwise3x3_kernel<2, 1><<<(unsigned)blocks, 256, 0, st>>>(p);
-    else if (i.stride == 1 && TQ == 1) depthwise3x3_kernel<1, 1><<<(unsigned)blocks, 256, 0, st>>>(p);
-    else if (i.stride == 2 && TQ == 2) depthwise3x3_kernel<2, 2><<<(unsigned)blocks, 256, 0, st>>>(p);
-    else if (i.stride == 2 && TQ == 1) depthwise3x3_kernel<1, 2><<<(unsigned)blocks, 256, 0, st>>>(p);
-    else return CPRUNE_ERR_INTERNAL;
+    dw_tile(i, &p.TH, &p.TW, &p.G);
+    p.IH = (p.TH - 1) * i.stride + 3;
+    p.IW = (p.TW - 1) * i.stride + 3;
+    p.tiles_h = (i.P + p.TH - 1) / p.TH;
+    p.tiles_w = (i.Q + p.TW - 1) / p.TW;
+    p.cblocks = (p.c8 + p.G - 1) / p.G;
+    p.status = device_status_word();
+    if (!p.status) return cuda_fail(cudaGetLastError(), "status word");
+    CUtensorMap tm;
+    {
+        std::lock_guard<std::mutex> lock(plan->mu);
+        if (plan->map_x != x) {
+            unsigned long long dims[4] = {(unsigned long long)i.c_pad, (unsigned long long)i.W, (unsigned long long)i.H,
+                                          (unsigned long long)i.N};
+            unsigned long long strides[3] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.W * i.c_pad * 2,
+                                             (unsigned long long)i.H * i.W * i.c_pad * 2};
+            unsigned box[4] = {(unsigned)(p.G * 8), (unsigned)p.IW, (unsigned)p.IH, 1};
+            cprune_status s = encode_tiled_bf16(&plan->tm_a, x, 4, dims, strides, box);
+            if (s != CPRUNE_OK) return s;
+            plan->map_x = x;
+        }
+        std::memcpy(&tm, &plan->tm_a, sizeof(CUtensorMap));
+    }
+    const long long blocks = (long long)i.N * p.tiles_h * p.tiles_w * p.cblocks;
+    if (blocks == 0) return CPRUNE_OK;
+    if (blocks > 0x7fffffffLL || p.IW > 256 || p.IH > 256) return CPRUNE_ERR_UNSUPPORTED;
+    const int smem = p.IH * p.IW * p.G * 16;
+    static std::mutex attr_mu;
+    static int attr_set = 0;
+    {
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (!attr_set) {
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(depthwise3x3_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(depthwise3x3_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+            attr_set = 1;
+        }
+    }
+    if (smem > 100 * 1024) return CPRUNE_ERR_UNSUPPORTED;
+    const int threads = ((p.TW * p.G + 31) / 32) * 32;
+    if (i.stride == 1) depthwise3x3_kernel<1><<<(unsigned)blocks, threads, smem, st>>>(tm, p);
+    else depthwise3x3_kernel<2><<<(unsigned)blocks, threads, smem, st>>>(tm, p);
     CPRUNE_LAUNCH_CHECK("depthwise3x3_kernel");
     return CPRUNE_OK;
 }

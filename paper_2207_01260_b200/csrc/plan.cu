@@ -46,8 +46,15 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     if (depthwise) {
         if (family != CPRUNE_KERNEL_AUTO && family != CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;
         family = CPRUNE_KERNEL_DEPTHWISE;
-        i.tile_m = 1;
-        i.tile_n = i.stride == 1 ? (i.Q >= 4 ? 4 : (i.Q >= 2 ? 2 : 1)) : (i.Q >= 2 ? 2 : 1);  // output columns per thread
+        // output pixels per CTA (rows x columns), see depthwise.cu
+        {
+            const int c8 = i.c_pad / 8, G = c8 < 8 ? c8 : 8;
+            int tw = 224 / G;
+            if (i.stride == 2 && tw > 28) tw = 28;
+            i.tile_n = i.Q < tw ? i.Q : tw;
+            const int th = i.stride == 1 ? 14 : (i.tile_n <= 14 ? 7 : 4);
+            i.tile_m = i.P < th ? i.P : th;
+        }
         i.tile_k = 8;
     } else {
         if (family == CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;

@@ -37,12 +37,15 @@ namespace cprune {
 cprune_status launch_conv_direct(const cprune_plan *plan, const void *x, const void *w, const float *b,
                                  const void *res, void *y, cudaStream_t st);
 // depthwise 3x3
-cprune_status launch_depthwise(const cprune_plan *plan, const void *x, const void *w, const float *b,
+cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, const float *b,
                                const void *res, void *y, cudaStream_t st);
 // tcgen05 implicit GEMM
 cprune_status plan_conv_tensor(cprune_plan *plan);  // fills tile fields of plan->info; UNSUPPORTED if not eligible
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
                                  void *y, cudaStream_t st);
+// tiled bf16 tensor map without swizzle, out-of-bounds elements read as zero
+cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
+                                const unsigned long long *strides_bytes, const unsigned *box);
 // 2x2 stride-2 max-pool as a separate pass (used when a plan asks for a pool and the conv kernel
 // does not fuse it): x [N][H][W][c] -> y [N][H/2][W/2][c]
 cprune_status launch_maxpool(const void *x, int N, int H, int W, int c_pad, int k, int stride, int pad, void *y,
