@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
 static void dw_tile(const cprune_plan_info &i, int *TH, int *TW, int *G) {
     const int c8 = i.c_pad / 8;
     *G = c8 < 8 ? c8 : 8;
-    int tw = 224 / *G;                      // about 224 threads per CTA
+    int tw = 112 / *G;                      // about 112 threads per CTA: small patches, several CTAs per SM
     if (i.stride == 2 && tw > 28) tw = 28;  // keeps the input patch small
     *TW = i.Q < tw ? i.Q : tw;
     int th = i.stride == 1 ? 14 : (*TW <= 14 ? 7 : 4);

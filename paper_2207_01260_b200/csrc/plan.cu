@@ -49,7 +49,7 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
         // output pixels per CTA (rows x columns), see depthwise.cu
         {
             const int c8 = i.c_pad / 8, G = c8 < 8 ? c8 : 8;
-            int tw = 224 / G;
+            int tw = 112 / G;
             if (i.stride == 2 && tw > 28) tw = 28;
             i.tile_n = i.Q < tw ? i.Q : tw;
             const int th = i.stride == 1 ? 14 : (i.tile_n <= 14 ? 7 : 4);
