@@ -13,7 +13,7 @@
 //               float32) with the accumulator in tensor memory; two accumulator buffers so
 //               that the epilogue of one tile overlaps the main loop of the next;
 //   warps 2..5  epilogue: tcgen05.ld the accumulator, bias (+ residual), activation, bf16,
-//               write 16-filter-wide sub-tiles into swizzled shared memory, TMA-store them to
+//               write 64-filter-wide sub-tiles into swizzled shared memory, TMA-store them to
 //               the NHWC output (the store clips rows beyond the last pixel and filters beyond
 //               k_pad by itself).
 // An MMA instruction costs about the same for any N up to 256, so the plan picks the orientation
@@ -41,7 +41,7 @@ constexpr int ACC_STRIDE = 256;    // column offset of the second accumulator bu
 constexpr int MAX_STAGES = 8;
 constexpr long long WAIT_LIMIT_CYCLES = 1LL << 31;   // about a second
 constexpr int ORIENT_PIX = 0, ORIENT_FILT = 1;
-constexpr int SUB = 16;            // filters per staged sub-tile (32-byte rows, 32-byte swizzle)
+constexpr int SUB = 64;            // filters per staged sub-tile (128-byte rows, 128-byte swizzle)
 constexpr int CTRL_BYTES = 2048;   // barriers, flags, bias vector
 constexpr int GROUP_BYTES = 16384; // one staging buffer (see the kernel)
 
@@ -213,9 +213,9 @@ __device__ __forceinline__ uint64_t smem_desc_interleaved(uint32_t addr, uint32_
     return d;
 }
 
-// Byte offset of (row, 16-byte half h) in a staged sub-tile of 32-byte rows under the 32-byte
-// swizzle (address bit 4 is XORed with bit 7, i.e. with bit 2 of the row).
-__device__ __forceinline__ uint32_t sub_off(int row, int h) { return (uint32_t)(row * 32 + ((h ^ ((row >> 2) & 1)) << 4)); }
+// Byte offset of (row, 16-byte chunk c of 8) in a staged sub-tile of 128-byte rows under the
+// 128-byte swizzle (address bits 4..6 are XORed with bits 7..9, i.e. with the row modulo 8).
+__device__ __forceinline__ uint32_t sub_off(int row, int c) { return (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)); }
 
 // ---------------------------------------------------------------------------------------- kernel
 
@@ -230,9 +230,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     uint8_t *smem = smem_raw + (base - raw);
     const int x_bytes = p.PT * BK * 2;                     // pixel operand of one stage
     const int stage_bytes = x_bytes + p.FT * BK * 2;
-    // staging buffers, each one group of sub-tiles [rows][16 filters] bf16:
-    //   ORIENT_PIX:  128 pixels x 64 filters  = 4 sub-tiles of 4 KB
-    //   ORIENT_FILT:  64 pixels x 128 filters = 8 sub-tiles of 2 KB
+    // staging buffers, each one group of sub-tiles [rows][64 filters] bf16:
+    //   ORIENT_PIX:  128 pixels x 64 filters  = 1 sub-tile of 16 KB
+    //   ORIENT_FILT:  64 pixels x 128 filters = 2 sub-tiles of 8 KB
     constexpr int GROUP_ROWS = ORIENT == ORIENT_PIX ? 128 : 64;
     constexpr int SUB_BYTES = GROUP_ROWS * SUB * 2;
     const uint32_t staging0 = base + (uint32_t)p.stages * stage_bytes;
@@ -461,7 +461,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     uint32_t v[64];
 #pragma unroll
                     for (int sb = 0; sb < 4; ++sb)
-                        if (cg + sb * SUB < p.FT) tmem_ld16(t_row + (uint32_t)(cg + sb * SUB), v + sb * 16);
+                        if (cg + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(cg + sb * 16), v + sb * 16);
                     tmem_ld_wait();
                     if (g == groups - 1) {               // accumulator fully read: hand it back to the MMA warp
                         tc_fence_before();
@@ -470,7 +470,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     }
 #pragma unroll
                     for (int sb = 0; sb < 4; ++sb) {
-                        const int c0 = cg + sb * SUB;
+                        const int c0 = cg + sb * 16;
                         if (c0 < p.FT) {
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
@@ -488,7 +488,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                 }
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], p.act);
-                                *(bf16x8 *)(buf_ptr + sb * SUB_BYTES + sub_off(trow, h)) = pack8(f);
+                                *(bf16x8 *)(buf_ptr + sub_off(trow, sb * 2 + h)) = pack8(f);
                             }
                         }
                     }
@@ -497,11 +497,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     ok = epi_sync();
                     if (!ok) break;
                     if (store_thread) {
-                        for (int sb = 0; sb < 4; ++sb) {
-                            const int c0 = cg + sb * SUB;
-                            if (c0 < p.FT && k_base + c0 < p.k_pad)
-                                tma_store_2d(&tm_y, buf + sb * SUB_BYTES, k_base + c0, (int)m0);
-                        }
+                        if (k_base + cg < p.k_pad) tma_store_2d(&tm_y, buf, k_base + cg, (int)m0);
                         tma_store_commit();
                     }
                     ++group_counter;
@@ -514,9 +510,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 const int n_sub = (p.k_pad + SUB - 1) / SUB;       // sub-tiles that hold real filters
                 const bool warp_has_work = quarter * 32 < p.k_pad; // all 32 filters of this warp may be padding
                 const int groups = p.PT / 64;
-                const int hk = (k >> 3) & 1;
+                const int hk = (k >> 3) & 7;              // 16-byte chunk of this filter within its 128-byte row
                 for (int g = 0; g < groups && ok; ++g) {
-                    uint8_t *dst = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 4) * SUB_BYTES + (k & 7) * 2;
+                    uint8_t *dst = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 6) * SUB_BYTES + (k & 7) * 2;
                     const uint32_t buf = staging0 + (group_counter & 1u) * GROUP_BYTES;
                     const long long mg = m0 + g * 64;
                     if (warp_has_work) {
@@ -676,12 +672,14 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
         tiles_n = (k16 + 255) / 256;
         while (true) {
             int next = tiles_n + 1;
-            int ft_next = round_up((k16 + next - 1) / next, 16);
+            int ft_next = round_up((k16 + next - 1) / next, 64);
             if (ft_next < 128) break;
             if ((long long)tiles_m * tiles_n >= 148) break;
             tiles_n = next;
         }
-        FT = round_up((k16 + tiles_n - 1) / tiles_n, 16);
+        // with several filter tiles every tile must end on a 64-filter boundary: the staged stores
+        // are 64 filters wide and only the tensor's own edge clips them
+        FT = round_up((k16 + tiles_n - 1) / tiles_n, tiles_n > 1 ? 64 : 16);
         tiles_n = (k16 + FT - 1) / FT;
     }
     int stages = MAX_STAGES;
@@ -740,14 +738,14 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         plan->map_w = w;
     }
     if (plan->map_y != y) {
-        // output as a 2-D tensor [pixels][k_pad]; stored in boxes of 16 filters x 128 or 64 pixels
+        // output as a 2-D tensor [pixels][k_pad]; stored in boxes of 64 filters x 128 or 64 pixels
         const long long M = (long long)i.N * i.P * i.Q;
         cuuint64_t dims[2] = {(cuuint64_t)i.k_pad, (cuuint64_t)M};
         cuuint64_t strides[1] = {(cuuint64_t)i.k_pad * 2};
         cuuint32_t box[2] = {SUB, (cuuint32_t)(plan->orient == ORIENT_PIX ? 128 : 64)};
         cuuint32_t estr[2] = {1, 1};
         CUresult r = g_encode_tiled(&plan->tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
-                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(y)");
         plan->map_y = y;
