@@ -26,6 +26,7 @@
 // released and the kernel returns.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -55,6 +56,10 @@ struct TcParams {
     int small_c;       // c_pad == 8 (3-channel stems): a 64-wide K block is 8 taps x 8 channels
     int iters;         // pipeline stages per tile (K blocks, plus residual blocks)
     int res_iters;     // ORIENT_FILT with a residual: trailing stages that add it on the tensor core
+    int splits;        // split-K: CTAs that share one output tile, each a slice of the K blocks
+    int ipp;           // K blocks per slice
+    int k_alloc;       // row length of the float32 partial sums
+    float *partial;    // [splits][M][k_alloc] when splits > 1
     const float *bias;
     const __nv_bfloat16 *res;
     int *status;
@@ -271,7 +276,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int total_tiles = p.tiles_m * p.tiles_n;
+    const int total_tiles = p.tiles_m * p.tiles_n * p.splits;   // work items: (tile, K slice), slice fastest
     const int PQ = p.P * p.Q;
 
     if (warp == 0) {
@@ -279,7 +284,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
+            const int tile = item / p.splits, split = item - tile * p.splits;
+            const int it_begin = split * p.ipp, it_end = min(p.iters, it_begin + p.ipp);
             const int mt = tile / p.tiles_n, nt_f = tile - mt * p.tiles_n;
             const long long m0 = (long long)mt * p.PT;
             const int n_img = (int)(m0 / PQ);
@@ -311,20 +318,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             } else {
-            for (int r = 0; r < p.R && ok; ++r)
-                for (int s = 0; s < p.S && ok; ++s)
-                    for (int cb = 0; cb < p.cblks; ++cb) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
-                        if (!ok) break;
-                        if (elect_one()) {
-                            const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
-                            mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
-                            tma_load_im2col(x_dst, &tm_x, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
-                            tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), cb * BK, r * p.S + s, nt_f * p.FT);
-                        }
-                        __syncwarp();
-                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-                    }
+            for (int it = it_begin; it < it_end - (p.splits == 1 ? p.res_iters : 0); ++it) {
+                const int tap = it / p.cblks, cb = it - tap * p.cblks;
+                const int r = tap / p.S, s = tap - r * p.S;
+                ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
+                    mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
+                    tma_load_im2col(x_dst, &tm_x, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
+                    tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), cb * BK, tap, nt_f * p.FT);
+                }
+                __syncwarp();
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+            }
             }
             // residual blocks (ORIENT_FILT): the residual tile [PT pixels][64 filters] is the pixel-side
             // operand and a 64-column slice of the identity matrix the filter-side operand, so that the
@@ -350,13 +357,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         int stage = 0, acc = 0;
         uint32_t phase = 0, acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
+            const int split = item % p.splits;
+            const int it_begin = split * p.ipp, it_end = min(p.iters, it_begin + p.ipp);
             ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_STRIDE);
             uint32_t accumulate = 0;
-            for (int it = 0; it < p.iters; ++it) {
+            for (int it = it_begin; it < it_end; ++it) {
                 ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag, p.status));
                 if (!ok) break;
                 const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
@@ -429,7 +438,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             epi_phase ^= 1u;
             return r;
         };
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
+            const int tile = item / p.splits, split = item - tile * p.splits;
             const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
             const long long m0 = (long long)mt * p.PT;
             const int k_base = nt * p.FT;
@@ -440,7 +450,43 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * ACC_STRIDE);
 
-            if (ORIENT == ORIENT_PIX) {
+            if (p.splits > 1) {
+                // split-K: this CTA holds a partial sum; store it as float32, the finalize kernel adds
+                // the slices in a fixed order and applies bias, residual and activation
+                float *part = p.partial + (size_t)split * (size_t)p.M * p.k_alloc;
+                if (ORIENT == ORIENT_PIX) {
+                    const long long m = m0 + trow;
+                    for (int c0 = 0; c0 < p.FT; c0 += 16) {
+                        uint32_t v[16];
+                        tmem_ld16(t_row + (uint32_t)c0, v);
+                        tmem_ld_wait();
+                        if (m < p.M) {
+                            float4 *dst = (float4 *)(part + (size_t)m * p.k_alloc + k_base + c0);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                        }
+                    }
+                } else {
+                    const int k = trow;
+                    if (quarter * 32 < p.k_pad) {
+                        for (int c0 = 0; c0 < p.PT; c0 += 16) {
+                            uint32_t v[16];
+                            tmem_ld16(t_row + (uint32_t)c0, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const long long m = m0 + c0 + j;
+                                if (m < p.M) part[(size_t)m * p.k_alloc + k] = __uint_as_float(v[j]);
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+            } else if (ORIENT == ORIENT_PIX) {
                 // rows = pixels, columns = filters; groups of 64 filters
                 const long long m = m0 + trow;
                 const bool row_ok = m < p.M;
@@ -599,6 +645,36 @@ static cprune_status load_driver_entry_points() {
     return CPRUNE_OK;
 }
 
+// Split-K finalize: y[m][k] = act(bias[k] + residual[m][k] + sum over slices of partial[s][m][k]),
+// slices added in index order (deterministic).  One thread per (pixel, 8 filters).
+__global__ void __launch_bounds__(256) splitk_finalize_kernel(const float *__restrict__ partial, int splits, long long M,
+                                                              int k_alloc, int k8, const float *__restrict__ bias,
+                                                              const bf16x8 *__restrict__ res, int act,
+                                                              bf16x8 *__restrict__ y) {
+    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= M * k8) return;
+    const long long m = e / k8;
+    const int kg = (int)(e - m * k8);
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = __ldg(bias + kg * 8 + j);
+    for (int sidx = 0; sidx < splits; ++sidx) {
+        const float4 *src = (const float4 *)(partial + ((size_t)sidx * M + m) * k_alloc + kg * 8);
+        const float4 a = __ldg(src), b = __ldg(src + 1);
+        f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+        f[4] += b.x; f[5] += b.y; f[6] += b.z; f[7] += b.w;
+    }
+    if (res) {
+        float rf[8];
+        unpack8(ldg8(res + e), rf);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] += rf[j];
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], act);
+    y[e] = pack8(f);
+}
+
 // 128 x 128 identity in bf16: the filter-side operand of the residual blocks (see the producer).
 static __device__ __align__(256) __nv_bfloat16 g_identity[128 * 128];
 
@@ -697,6 +773,34 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     if (plan->small_c) i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * ((i.R * i.S + 1) / 2) * 16.0;
     plan->staging_bufs = bufs;
     plan->smem_bytes = smem_for(stages, PT, FT, bufs, group_rows);
+    // Split-K when the tiles cannot fill the SMs: slices of the K blocks go to different CTAs, which
+    // store float32 partial sums; a small second kernel adds them.  The choice minimises a cost model
+    // fitted to measurements on B200 (microseconds): waves x (K blocks per slice x time per block +
+    // per-item overhead) + launch floor (+ the second pass).
+    plan->splits = 1;
+    const int iters = i.R * i.S * cblks;
+    const long long tiles = (long long)i.tiles_m * tiles_n;
+    if (!plan->small_c && tiles <= 100 && iters >= 4) {
+        const double blk = plan->orient == ORIENT_PIX ? (FT > 128 ? 0.375 * FT / 128.0 : 0.375) : 0.45;
+        auto cost = [&](int sp) {
+            const int ipp = (iters + sp - 1) / sp;
+            return (double)ceil_div(tiles * sp, 148) * (ipp * blk + 4.0) + 6.0 + (sp > 1 ? 2.5 : 0.0);
+        };
+        double best = cost(1);
+        for (int sp = 2; sp <= 16 && sp * 2 <= iters; ++sp) {
+            const int ipp = (iters + sp - 1) / sp;
+            if ((sp - 1) * ipp >= iters) continue;              // a slice would be empty
+            if ((double)sp * M * i.k_alloc * 4.0 > 256e6) break; // keep the partial sums within L2 reach
+            const double t = cost(sp);
+            if (t < best * 0.9) { best = t; plan->splits = sp; }
+        }
+    }
+    if (const char *force = getenv("CPRUNE_FORCE_SPLITS")) {   // measurement override
+        int sp = atoi(force);
+        if (sp >= 1 && !plan->small_c && sp <= iters && (sp - 1) * ((iters + sp - 1) / sp) < iters) plan->splits = sp;
+    }
+    plan->ipp = (iters + plan->splits - 1) / plan->splits;
+    plan->partial_bytes = plan->splits > 1 ? (size_t)plan->splits * (size_t)M * i.k_alloc * 4 : 0;
     return CPRUNE_OK;
 }
 
@@ -787,10 +891,12 @@ static int sm_count() {
 }
 
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
-                                 void *y, cudaStream_t st) {
+                                 void *y, void *partial, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
     CUtensorMap tm_x, tm_w, tm_y, tm_res, tm_id;
-    const bool mma_res = plan->orient == ORIENT_FILT && res != nullptr;
+    const bool split = plan->splits > 1;
+    if (split && !partial) return CPRUNE_ERR_INVALID_ARG;
+    const bool mma_res = plan->orient == ORIENT_FILT && res != nullptr && !split;
     {
         std::lock_guard<std::mutex> lock(plan->mu);
         if (plan->map_x != x || plan->map_w != w || plan->map_y != y || (mma_res && plan->map_res != res)) {
@@ -821,14 +927,19 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     p.ksteps_last = (i.c_pad - (p.cblks - 1) * BK + 15) / 16;
     p.PT = i.tile_m; p.FT = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
     p.small_c = plan->small_c;
+    p.splits = plan->splits;
+    p.ipp = plan->ipp;
+    p.k_alloc = i.k_alloc;
+    p.partial = (float *)partial;
     p.res_iters = mma_res ? (i.k_pad + BK - 1) / BK : 0;
     p.iters = (plan->small_c ? (i.R * i.S + 7) / 8 : i.R * i.S * p.cblks) + p.res_iters;
+    if (plan->splits == 1) p.ipp = p.iters;   // one slice covers everything, the residual blocks included
     p.act = plan->opts.activation;
     p.bias = b;
-    p.res = mma_res ? nullptr : (const __nv_bfloat16 *)res;   // ORIENT_PIX adds it in the epilogue
+    p.res = (mma_res || split) ? nullptr : (const __nv_bfloat16 *)res;   // ORIENT_PIX adds it in the epilogue
     p.status = device_status_word();
     if (!p.status) return cuda_fail(cudaGetLastError(), "status word");
-    const int total = i.tiles_m * i.tiles_n;
+    const int total = i.tiles_m * i.tiles_n * plan->splits;
     if (total == 0) return CPRUNE_OK;
     const int grid = total < sm_count() ? total : sm_count();
     if (plan->orient == ORIENT_PIX)
@@ -836,6 +947,13 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     else
         conv_tc_kernel<ORIENT_FILT><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
     CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
+    if (split) {
+        const long long elems = p.M * (i.k_pad / 8);
+        splitk_finalize_kernel<<<(unsigned)ceil_div(elems, 256), 256, 0, st>>>((const float *)partial, plan->splits, p.M,
+                                                                              i.k_alloc, i.k_pad / 8, b, (const bf16x8 *)res,
+                                                                              plan->opts.activation, (bf16x8 *)y);
+        CPRUNE_LAUNCH_CHECK("splitk_finalize_kernel");
+    }
     return CPRUNE_OK;
 }
 

@@ -77,7 +77,9 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     const double rs = (double)i.R * i.S;
     i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * i.S * i.c_pad * 2;
     i.packed_bias_bytes = (size_t)i.k_alloc * sizeof(float);
-    i.workspace_bytes = pl->opts.pool == CPRUNE_POOL_MAX2X2 ? (size_t)i.N * i.P * i.Q * i.k_pad * 2 : 0;
+    // workspace: [unpooled conv output if a pool follows][split-K partial sums]
+    pl->pool_bytes = pl->opts.pool == CPRUNE_POOL_MAX2X2 ? ((size_t)i.N * i.P * i.Q * i.k_pad * 2 + 255) / 256 * 256 : 0;
+    i.workspace_bytes = pl->pool_bytes + (family == CPRUNE_KERNEL_TENSOR ? pl->partial_bytes : 0);
     i.algorithmic_bytes = 2.0 * ((double)i.N * i.H * i.W * i.C + (double)i.N * i.out_h * i.out_w * i.K +
                                  (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
                                  (double)i.K * (i.C / i.groups) * rs) + 4.0 * i.K;
@@ -175,12 +177,13 @@ cprune_status cprune_task_run(cprune_plan *plan, const void *x, const void *w_pa
         return CPRUNE_ERR_INVALID_ARG;
     const cprune_plan_info &i = plan->info;
     const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
-    if (pool && !workspace) return CPRUNE_ERR_INVALID_ARG;
+    if (i.workspace_bytes && !workspace) return CPRUNE_ERR_INVALID_ARG;
     void *conv_out = pool ? workspace : y;
+    void *partial = plan->partial_bytes ? (void *)((char *)workspace + plan->pool_bytes) : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
     cprune_status s;
     switch (i.kernel) {
-        case CPRUNE_KERNEL_TENSOR: s = launch_conv_tensor(plan, x, w_packed, b_packed, residual, conv_out, st); break;
+        case CPRUNE_KERNEL_TENSOR: s = launch_conv_tensor(plan, x, w_packed, b_packed, residual, conv_out, partial, st); break;
         case CPRUNE_KERNEL_DIRECT: s = launch_conv_direct(plan, x, w_packed, b_packed, residual, conv_out, st); break;
         case CPRUNE_KERNEL_DEPTHWISE: s = launch_depthwise(plan, x, w_packed, b_packed, residual, conv_out, st); break;
         default: return CPRUNE_ERR_INTERNAL;

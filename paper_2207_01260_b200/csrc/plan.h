@@ -28,6 +28,10 @@ struct cprune_plan {
     int smem_bytes = 0;
     int orient = 0;                 // which side of the MMA the pixels are on
     int staging_bufs = 2;
+    int splits = 1;                 // split-K slices per output tile
+    int ipp = 0;                    // K blocks per slice
+    size_t pool_bytes = 0;          // unpooled conv output in the workspace when a 2x2 pool follows
+    size_t partial_bytes = 0;       // float32 partial sums in the workspace
     int small_c = 0;                // 3-channel stems: 8 taps x 8 channels per K block
 };
 
@@ -42,7 +46,7 @@ cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, 
 // tcgen05 implicit GEMM
 cprune_status plan_conv_tensor(cprune_plan *plan);  // fills tile fields of plan->info; UNSUPPORTED if not eligible
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
-                                 void *y, cudaStream_t st);
+                                 void *y, void *partial, cudaStream_t st);
 // tiled bf16 tensor map without swizzle, out-of-bounds elements read as zero
 cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
                                 const unsigned long long *strides_bytes, const unsigned *box);
