@@ -28,6 +28,10 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+# DRAM bytes (read + write) of all conv_tc_kernel launches of one model pass, from the ncu capture summarised in
+# profiles/conv_tc_resnet18_b64_dram_traffic.md; None where no capture of the current kernel exists.
+CONV_TC_DRAM_BYTES_PER_STEP = {"resnet18": 415.9e6, "mobilenet_v2": None, "vgg16_cifar": None}
+
 WORKLOADS = {"resnet18": ("resnet18", 64), "mobilenet_v2": ("mobilenet_v2", 64), "vgg16_cifar": ("vgg16_cifar", 128)}
 
 
@@ -86,6 +90,23 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, device=None):
+    """Every rank passes its own timings; all get the element-wise maximum (the slowest replica
+    decides).  Without an initialised process group the values come back unchanged."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def replica_seed(base_seed: int, rank: int) -> int:
+    """Seed of the input batch of replica `rank`: replicas process different images."""
+    return base_seed + 17 * rank
+
+
 def cpu_reference(args, table_name, batch):
     """The oracle, as it stands, on the host cores: each step runs the pruned network on a bounded
     sample of the batch."""
@@ -115,11 +136,21 @@ def main():
     ap.add_argument("--workload", default="resnet18", choices=sorted(WORKLOADS))
     ap.add_argument("--no-graph", action="store_true", help="enqueue every launch from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-task-times", action="store_true",
+                    help="skip the per-task timing passes (and with them the roofline object); for profiler launch lists")
     ap.add_argument("--task", default=None,
                     help="time ONE conv task instead of a model: N,C,H,W,K,R,stride,pad[,groups[,act[,residual]]]")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every distinct conv shape of the four models while the kept filter count K goes "
+                         "from full width down to a quarter (the staircase of latency against K)")
+    ap.add_argument("--sweep-stride", type=int, default=0, help="step in K (0: about 24 points per shape; 1: every K)")
+    ap.add_argument("--sweep-batch", type=int, default=64)
+    ap.add_argument("--sweep-out", default="sweep.jsonl")
     args = ap.parse_args()
     if args.task:
         return task_bench(args)
+    if args.sweep:
+        return sweep_bench(args)
     table_name, batch = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -163,7 +194,7 @@ def main():
 
     table = wl.MODELS[table_name]()
     weights = wl.model_weights(table)
-    x_host = torch.from_numpy(wl.model_input(table, batch, seed=table["seed"] + 17 * rank)).pin_memory()
+    x_host = torch.from_numpy(wl.model_input(table, batch, seed=replica_seed(table["seed"], rank))).pin_memory()
 
     t0 = time.perf_counter()
     net = PrunedNetwork(table, weights, batch, device=dev)
@@ -198,30 +229,26 @@ def main():
     clocks = sampler.stop()
     cp.cprune_poll_device_status()
 
-    # ---------------- end to end: pinned host input -> device -> model -> logits back on the host
+    # ---------------- end to end: pinned host input -> device -> model -> logits back on the host, all inside
+    # the C-ABI call cprune_model_run_host (copy of step i+1 overlaps the kernels of step i)
     for _ in range(3):
-        x.copy_(x_host, non_blocking=True)
-        net.run(x, logits, use_graph)
-        logits_host.copy_(logits, non_blocking=True)
+        net.run_host(x_host, logits_host)
     barrier()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record(stream)
     for _ in range(args.steps):
-        x.copy_(x_host, non_blocking=True)
-        net.run(x, logits, use_graph)
-        logits_host.copy_(logits, non_blocking=True)
+        net.run_host(x_host, logits_host)
     e3.record(stream)
     barrier()
     ms_e2e = e2.elapsed_time(e3)
+    if rank == 0 and not torch.equal(logits_host, logits.cpu()):
+        raise RuntimeError("host-buffer path and device path disagree")
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev if world > 1 else None)
 
     # ---------------- per-task timing of the tensor-core kernel (roofline of the dominant kernel)
     roof, per_task = None, []
-    if rank == 0:
+    if rank == 0 and not args.no_task_times:
         peaks = measured_peaks()
         per_task = net_task_times(cp, net, table, x, reps=5)
         tens = [t for t in per_task if t["kernel"] == "tensor"]
@@ -237,7 +264,10 @@ def main():
             tf = sum(t["flops"] for t in tens) / 1e12
             ach = tf / (t_tens * 1e-3)
             roof = {"kernel": "conv_tc_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None,
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                    "traffic": CONV_TC_DRAM_BYTES_PER_STEP.get(args.workload),
+                    "traffic_note": "DRAM bytes of all launches of this kernel in one step (ncu); algorithmic bytes alongside",
+                    "algorithmic_bytes": sum(t["bytes"] for t in tens),
                     "peak_source": peaks["source"] + " (sustained bf16 GEMM)", "launches_per_step": len(tens),
                     "ms_per_step": t_tens}
 
@@ -338,6 +368,74 @@ def task_bench(args):
             "buffer_sets": nsets, "tile_n": i["tile_n"], "tiles": i["tiles_m"] * i["tiles_n"], "stages": i["stages"],
             "steps": args.steps, "padded_flops_ratio": i["padded_flops"] / i["flops"]}
     print(json.dumps(line))
+
+
+def sweep_bench(args):
+    """Latency and TFLOP/s (or GB/s) of every distinct conv shape against the kept filter count."""
+    import torch
+
+    import paper_2207_01260_b200 as cp
+    import workloads as wl
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    N = args.sweep_batch
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    out = open(args.sweep_out, "w")
+    npoints, t0 = 0, time.perf_counter()
+    worst = {}
+    for shp in wl.sweep_shapes():
+        dw = shp["groups"] > 1
+        kfull = shp["K"]
+        stride = args.sweep_stride or max(1, (kfull - (kfull + 3) // 4) // 24)
+        ks = list(range(kfull, (kfull + 3) // 4 - 1, -stride))
+        for K in ks:
+            C = K if dw else shp["C"]
+            plan = cp.cprune_task_plan(N, C, shp["H"], shp["W"], K, shp["R"], shp["S"], shp["stride"], shp["pad"],
+                                       K if dw else 1, shp["act"])
+            i = plan.info
+            x = torch.randn((N, shp["H"], shp["W"], i["c_pad"]), device="cuda", generator=gen).to(torch.bfloat16)
+            if i["c_pad"] > C:
+                x[..., C:] = 0
+            w = torch.randn((K, 1 if dw else C, shp["R"], shp["S"]), device="cuda", generator=gen) * (2.0 / (shp["R"] * shp["S"] * (1 if dw else C))) ** 0.5
+            wp, bp = cp.cprune_pack_weights(plan, w.contiguous(), torch.zeros(K, device="cuda"))
+            y = torch.empty((N, i["out_h"], i["out_w"], i["k_pad"]), dtype=torch.bfloat16, device="cuda")
+            ws = torch.empty(max(i["workspace_bytes"], 16), dtype=torch.uint8, device="cuda")
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            reps = 10
+            with torch.cuda.stream(side):
+                cp.cprune_task_run(plan, x, wp, bp, None, y, ws)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(graph, stream=side):
+                    for _ in range(reps):
+                        cp.cprune_task_run(plan, x, wp, bp, None, y, ws)
+            graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            tf = i["flops"] / ms / 1e9
+            gbs = i["algorithmic_bytes"] / ms / 1e6
+            ai = i["flops"] / i["algorithmic_bytes"]
+            bound = "tensor" if ai > peaks["bf16_tflops_sustained"] * 1e3 / peaks["hbm_gbs"] else "hbm"
+            frac = tf / peaks["bf16_tflops_sustained"] if bound == "tensor" else gbs / peaks["hbm_gbs"]
+            rec = {"model": shp["model"], "layer": shp["layer"], "N": N, "C": C, "K": K, "H": shp["H"], "W": shp["W"],
+                   "R": shp["R"], "stride": shp["stride"], "depthwise": dw, "kernel": cp.KERNEL_NAMES[i["kernel"]],
+                   "ms": ms, "tflops": tf, "gbs": gbs, "bound": bound, "frac": frac, "tile": [i["tile_m"], i["tile_n"]],
+                   "tiles": i["tiles_m"] * i["tiles_n"], "k_alloc": i["k_alloc"], "warm_l2": True}
+            out.write(json.dumps(rec) + "\n")
+            npoints += 1
+            key = (shp["model"], shp["layer"])
+            worst[key] = min(worst.get(key, 1e9), frac)
+        cp.cprune_poll_device_status()
+    out.close()
+    print(json.dumps({"metric": "conv_task_sweep", "points": npoints, "batch": N, "seconds": time.perf_counter() - t0,
+                      "out": args.sweep_out, "min_frac_over_shapes": min(worst.values()),
+                      "median_of_min_frac": float(np.median(list(worst.values())))}))
 
 
 def net_task_times(cp, net, table, x, reps=5):

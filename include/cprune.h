@@ -210,6 +210,13 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
  * task on `stream`.  With use_graph != 0 the launch sequence is captured into a CUDA graph on the first
  * call for a given (x, logits, stream) and replayed afterwards. */
 cprune_status cprune_model_run(cprune_model *model, const float *x, float *logits, int use_graph, void *stream);
+/* The same through HOST buffers: x_host float32 [N][H][W][C] and logits_host float32 [N][classes]
+ * (pinned memory makes the copies asynchronous).  The call enqueues the host-to-device copy on a
+ * private copy stream, the captured launch sequence and the device-to-host copy of the logits on
+ * `stream`, and returns without waiting; synchronise `stream` before reading logits_host, and keep
+ * x_host unchanged until then.  Two device-side input buffers alternate, so the copy of one call
+ * overlaps the kernels of the previous one.  The first call allocates those buffers (cudaMalloc). */
+cprune_status cprune_model_run_host(cprune_model *model, const float *x_host, float *logits_host, void *stream);
 /* Device pointer and element count of tensor `id` of the model (for tests). */
 cprune_status cprune_model_tensor(const cprune_model *model, int id, const void **ptr, int *n, int *h, int *w, int *c_pad);
 /* Copies tensor `id` (bf16 [n][h][w][c_pad]) into dst (device) on `stream`. */

@@ -26,7 +26,7 @@ EXPORTS = [
     "cprune_select_filters", "cprune_select_filters_static", "cprune_gather_rows", "cprune_gather_columns", "cprune_task_plan", "cprune_plan_query",
     "cprune_plan_release", "cprune_cache_clear", "cprune_cache_stats", "cprune_pack_weights", "cprune_task_run",
     "cprune_cast_input", "cprune_widen_output", "cprune_maxpool", "cprune_global_avgpool", "cprune_fc_pack",
-    "cprune_fc", "cprune_model_create", "cprune_model_run", "cprune_model_tensor", "cprune_model_copy_tensor", "cprune_model_launches",
+    "cprune_fc", "cprune_model_create", "cprune_model_run", "cprune_model_run_host", "cprune_model_tensor", "cprune_model_copy_tensor", "cprune_model_launches",
     "cprune_model_destroy", "cprune_poll_device_status",
 ]
 
@@ -93,6 +93,7 @@ def lib():
         L.cprune_fc.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p]
         L.cprune_model_create.argtypes = [c_int, c_int, c_int, c_int, POINTER(TaskDesc), c_int, POINTER(c_void_p)]
         L.cprune_model_run.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p]
+        L.cprune_model_run_host.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p]
         L.cprune_model_tensor.argtypes = [c_void_p, c_int, POINTER(c_void_p), POINTER(c_int), POINTER(c_int),
                                           POINTER(c_int), POINTER(c_int)]
         L.cprune_model_copy_tensor.argtypes = [c_void_p, c_int, c_void_p, c_void_p]
@@ -370,6 +371,16 @@ def cprune_model_run(model: Model, x, logits=None, use_graph=False, stream=None)
     _check(lib().cprune_model_run(model.handle, _ptr(x), _ptr(logits), 1 if use_graph else 0, _stream(stream)),
            "cprune_model_run")
     return logits
+
+
+def cprune_model_run_host(model: Model, x_host, logits_host, stream=None):
+    """x_host float32 [N,H,W,C] and logits_host float32 [N, classes] are HOST tensors (pinned for async
+    copies).  Returns immediately; synchronise the stream before reading logits_host."""
+    assert not x_host.is_cuda and not logits_host.is_cuda and x_host.dtype == torch.float32
+    assert x_host.is_contiguous() and logits_host.is_contiguous() and logits_host.dtype == torch.float32
+    _check(lib().cprune_model_run_host(model.handle, _ptr(x_host), _ptr(logits_host), _stream(stream)),
+           "cprune_model_run_host")
+    return logits_host
 
 
 def cprune_poll_device_status(stream=None):

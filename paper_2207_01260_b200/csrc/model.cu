@@ -23,11 +23,21 @@ struct cprune_model {
     size_t workspace_bytes = 0;
     int classes = 0;
     int launches = 0;
-    cudaGraphExec_t exec = nullptr;
-    const float *graph_x = nullptr;
-    float *graph_logits = nullptr;
-    cudaStream_t graph_stream = nullptr;
+    // captured launch sequences: slot 2 serves cprune_model_run, slots 0 and 1 the two device-side
+    // input buffers of cprune_model_run_host
+    struct GraphSlot {
+        cudaGraphExec_t exec = nullptr;
+        const float *x = nullptr;
+        float *logits = nullptr;
+        cudaStream_t stream = nullptr;
+    } graphs[3];
     cudaStream_t capture_stream = nullptr;   // private stream the launch sequence is recorded on
+    // host-buffer path: double-buffered device copies of the input and of the logits
+    float *host_x[2] = {nullptr, nullptr};
+    float *host_logits[2] = {nullptr, nullptr};
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copied[2] = {nullptr, nullptr}, done[2] = {nullptr, nullptr};
+    unsigned long long host_calls = 0;
 };
 
 namespace cprune {
@@ -112,7 +122,7 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
                 }
                 o.h = i.out_h; o.w = i.out_w; o.c = i.K;
                 if (i.workspace_bytes > m->workspace_bytes) m->workspace_bytes = i.workspace_bytes;
-                m->launches += d.plan->opts.pool ? 2 : 1;
+                m->launches += (d.plan->opts.pool ? 2 : 1) + (d.plan->splits > 1 ? 1 : 0);
                 break;
             }
             case CPRUNE_OP_MAXPOOL:
@@ -160,15 +170,13 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
     return CPRUNE_OK;
 }
 
-cprune_status cprune_model_run(cprune_model *m, const float *x, float *logits, int use_graph, void *stream) {
-    if (!m || !x || !logits) return CPRUNE_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (!use_graph) return enqueue(m, x, logits, st);
-    if (m->exec && m->graph_x == x && m->graph_logits == logits && m->graph_stream == st) {
-        CPRUNE_CUDA_CHECK(cudaGraphLaunch(m->exec, st));
+static cprune_status run_graph(cprune_model *m, int slot, const float *x, float *logits, cudaStream_t st) {
+    cprune_model::GraphSlot &g = m->graphs[slot];
+    if (g.exec && g.x == x && g.logits == logits && g.stream == st) {
+        CPRUNE_CUDA_CHECK(cudaGraphLaunch(g.exec, st));
         return CPRUNE_OK;
     }
-    if (m->exec) { cudaGraphExecDestroy(m->exec); m->exec = nullptr; }
+    if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
     // first call for this (x, logits, stream): run eagerly (this also encodes tensor maps and sets
     // kernel attributes outside of any capture), then record the same sequence for later replays
     cprune_status s = enqueue(m, x, logits, st);
@@ -182,10 +190,46 @@ cprune_status cprune_model_run(cprune_model *m, const float *x, float *logits, i
     cudaError_t e = cudaStreamEndCapture(m->capture_stream, &graph);
     if (s != CPRUNE_OK) { if (graph) cudaGraphDestroy(graph); return s; }
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
-    e = cudaGraphInstantiate(&m->exec, graph, 0);
+    e = cudaGraphInstantiate(&g.exec, graph, 0);
     cudaGraphDestroy(graph);
-    if (e != cudaSuccess) { m->exec = nullptr; return cuda_fail(e, "cudaGraphInstantiate"); }
-    m->graph_x = x; m->graph_logits = logits; m->graph_stream = st;
+    if (e != cudaSuccess) { g.exec = nullptr; return cuda_fail(e, "cudaGraphInstantiate"); }
+    g.x = x; g.logits = logits; g.stream = st;
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_model_run(cprune_model *m, const float *x, float *logits, int use_graph, void *stream) {
+    if (!m || !x || !logits) return CPRUNE_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!use_graph) return enqueue(m, x, logits, st);
+    return run_graph(m, 2, x, logits, st);
+}
+
+cprune_status cprune_model_run_host(cprune_model *m, const float *x_host, float *logits_host, void *stream) {
+    if (!m || !x_host || !logits_host) return CPRUNE_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t x_bytes = (size_t)m->N * m->H * m->W * m->C * sizeof(float);
+    const size_t l_bytes = (size_t)m->N * m->classes * sizeof(float);
+    if (!m->copy_stream) {   // first call: set up the two device-side buffer pairs (allocates)
+        CPRUNE_CUDA_CHECK(cudaStreamCreateWithFlags(&m->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CPRUNE_CUDA_CHECK(cudaMalloc((void **)&m->host_x[i], x_bytes));
+            CPRUNE_CUDA_CHECK(cudaMalloc((void **)&m->host_logits[i], l_bytes));
+            CPRUNE_CUDA_CHECK(cudaEventCreateWithFlags(&m->copied[i], cudaEventDisableTiming));
+            CPRUNE_CUDA_CHECK(cudaEventCreateWithFlags(&m->done[i], cudaEventDisableTiming));
+        }
+    }
+    const int slot = (int)(m->host_calls & 1);
+    // the copy of this call's input may overlap the previous call's kernels; it only has to wait
+    // until the call before that one has finished with the same device buffer
+    if (m->host_calls >= 2) CPRUNE_CUDA_CHECK(cudaStreamWaitEvent(m->copy_stream, m->done[slot], 0));
+    CPRUNE_CUDA_CHECK(cudaMemcpyAsync(m->host_x[slot], x_host, x_bytes, cudaMemcpyHostToDevice, m->copy_stream));
+    CPRUNE_CUDA_CHECK(cudaEventRecord(m->copied[slot], m->copy_stream));
+    CPRUNE_CUDA_CHECK(cudaStreamWaitEvent(st, m->copied[slot], 0));
+    cprune_status s = run_graph(m, slot, m->host_x[slot], m->host_logits[slot], st);
+    if (s != CPRUNE_OK) return s;
+    CPRUNE_CUDA_CHECK(cudaMemcpyAsync(logits_host, m->host_logits[slot], l_bytes, cudaMemcpyDeviceToHost, st));
+    CPRUNE_CUDA_CHECK(cudaEventRecord(m->done[slot], st));
+    ++m->host_calls;
     return CPRUNE_OK;
 }
 
@@ -214,8 +258,16 @@ int cprune_model_launches(const cprune_model *m) { return m ? m->launches : 0; }
 
 cprune_status cprune_model_destroy(cprune_model *m) {
     if (!m) return CPRUNE_ERR_INVALID_ARG;
-    if (m->exec) cudaGraphExecDestroy(m->exec);
+    for (auto &g : m->graphs)
+        if (g.exec) cudaGraphExecDestroy(g.exec);
     if (m->capture_stream) cudaStreamDestroy(m->capture_stream);
+    if (m->copy_stream) cudaStreamDestroy(m->copy_stream);
+    for (int i = 0; i < 2; ++i) {
+        if (m->host_x[i]) cudaFree(m->host_x[i]);
+        if (m->host_logits[i]) cudaFree(m->host_logits[i]);
+        if (m->copied[i]) cudaEventDestroy(m->copied[i]);
+        if (m->done[i]) cudaEventDestroy(m->done[i]);
+    }
     if (m->arena) cudaFree(m->arena);
     if (m->workspace) cudaFree(m->workspace);
     delete m;

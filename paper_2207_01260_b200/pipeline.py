@@ -129,6 +129,10 @@ class PrunedNetwork:
         """x: float32 [batch, H, W, C] device tensor -> float32 logits [batch, classes]."""
         return B.cprune_model_run(self.model, x, logits, use_graph)
 
+    def run_host(self, x_host, logits_host):
+        """Host buffers in and out (see cprune_model_run_host); asynchronous."""
+        return B.cprune_model_run_host(self.model, x_host, logits_host)
+
     def activation(self, name):
         """Copy of a stored activation as float32 numpy [N, h, w, c] without the pad lanes."""
         c = self.shapes[name][2]

@@ -273,6 +273,14 @@ def model_parity(cp, name, batch, hw=None, kernel="auto"):
     cp.cprune_poll_device_status()
     got = logits.cpu().numpy()
     assert np.array_equal(got, logits2.cpu().numpy()) and np.array_equal(got, logits3.cpu().numpy())
+    # the host-buffer entry point (copies inside the call, two alternating device buffers)
+    xh = torch.from_numpy(np.ascontiguousarray(x)).pin_memory()
+    lh = torch.empty(got.shape, dtype=torch.float32).pin_memory()
+    for _ in range(3):
+        net.run_host(xh, lh)
+    torch.cuda.synchronize()
+    cp.cprune_poll_device_status()
+    assert np.array_equal(lh.numpy(), got)
     matched = oracle.model_ref(table, pw, x, matched=True)
     exact = oracle.model_ref(table, pw, x, matched=False)
     rel = np.linalg.norm(got - matched) / np.linalg.norm(matched)
