@@ -165,9 +165,23 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
 }
 
 // Tile of output pixels per CTA and channel groups per CTA.
+// Channel groups (of 8 channels) per CTA: between 4 and 9, whichever wastes the fewest lanes in
+// the last channel block (c_pad/8 = 18 -> 9, 14 -> 7, 4 -> 4); larger wins ties.
+static int dw_groups(int c8) {
+    if (c8 <= 9) return c8;
+    int best = 8;
+    double best_util = 0.0;
+    for (int g = 9; g >= 4; --g) {
+        const double util = (double)c8 / (double)(((c8 + g - 1) / g) * g);
+        if (util > best_util + 1e-9) { best_util = util; best = g; }
+    }
+    return best;
+}
+
+// Tile of output pixels per CTA and channel groups per CTA.
 static void dw_tile(const cprune_plan_info &i, int *TH, int *TW, int *G) {
     const int c8 = i.c_pad / 8;
-    *G = c8 < 8 ? c8 : 8;
+    *G = dw_groups(c8);
     int tw = 112 / *G;                      // about 112 threads per CTA: small patches, several CTAs per SM
     if (i.stride == 2 && tw > 28) tw = 28;  // keeps the input patch small
     *TW = i.Q < tw ? i.Q : tw;

@@ -46,15 +46,9 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     if (depthwise) {
         if (family != CPRUNE_KERNEL_AUTO && family != CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;
         family = CPRUNE_KERNEL_DEPTHWISE;
-        // output pixels per CTA (rows x columns), see depthwise.cu
-        {
-            const int c8 = i.c_pad / 8, G = c8 < 8 ? c8 : 8;
-            int tw = 112 / G;
-            if (i.stride == 2 && tw > 28) tw = 28;
-            i.tile_n = i.Q < tw ? i.Q : tw;
-            const int th = i.stride == 1 ? 14 : (i.tile_n <= 14 ? 7 : 4);
-            i.tile_m = i.P < th ? i.P : th;
-        }
+        // output pixels per CTA (rows x columns) are chosen at launch, see depthwise.cu
+        i.tile_m = i.stride == 1 ? 14 : 4;
+        i.tile_n = 14;
         i.tile_k = 8;
     } else {
         if (family == CPRUNE_KERNEL_DEPTHWISE) st = CPRUNE_ERR_UNSUPPORTED;
