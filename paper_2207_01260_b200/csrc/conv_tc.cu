@@ -45,6 +45,7 @@ constexpr int ORIENT_PIX = 0, ORIENT_FILT = 1;
 constexpr int SUB = 64;            // filters per staged sub-tile (128-byte rows, 128-byte swizzle)
 constexpr int CTRL_BYTES = 2048;   // barriers, flags, bias vector
 constexpr int GROUP_BYTES = 16384; // one staging buffer (see the kernel)
+constexpr int POOL_SUB_BYTES = 16 * 128;   // pooled sub-tile of the filter-major orientation: 16 pixels x 64 filters
 
 struct TcParams {
     long long M;
@@ -56,6 +57,7 @@ struct TcParams {
     int small_c;       // c_pad == 8 (3-channel stems): a 64-wide K block is 8 taps x 8 channels
     int iters;         // pipeline stages per tile (K blocks, plus residual blocks)
     int res_iters;     // ORIENT_FILT with a residual: trailing stages that add it on the tensor core
+    int pool;          // 1: 2x2 stride-2 max-pool fused into the epilogue (tm_y then maps the pooled output)
     int splits;        // split-K: CTAs that share one output tile, each a slice of the K blocks
     int ipp;           // K blocks per slice
     int k_alloc;       // row length of the float32 partial sums
@@ -222,9 +224,22 @@ __device__ __forceinline__ uint64_t smem_desc_interleaved(uint32_t addr, uint32_
 // 128-byte swizzle (address bits 4..6 are XORed with bits 7..9, i.e. with the row modulo 8).
 __device__ __forceinline__ uint32_t sub_off(int row, int c) { return (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)); }
 
+// 2x2 stride-2 max-pool of 64 consecutive pixels (rows of Q pixels, Q a power of two <= 32) held by one
+// thread for one filter: 16 pooled values, written to rows 0..15 of a staged sub-tile.
+template <int Q>
+__device__ __forceinline__ void store_pooled(const float *f, uint8_t *dst, int chunk) {
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+        const int rp = t / (Q / 2), cq = t % (Q / 2);
+        const int b = rp * 2 * Q + 2 * cq;
+        const float m = fmaxf(fmaxf(f[b], f[b + 1]), fmaxf(f[b + Q], f[b + Q + 1]));
+        *(__nv_bfloat16 *)(dst + sub_off(t, chunk)) = __float2bfloat16_rn(m);
+    }
+}
+
 // ---------------------------------------------------------------------------------------- kernel
 
-template <int ORIENT>
+template <int ORIENT, int POOL>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res,
@@ -534,7 +549,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                 }
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], p.act);
-                                *(bf16x8 *)(buf_ptr + sub_off(trow, sb * 2 + h)) = pack8(f);
+                                if (POOL) {
+                                    // the 2x2 window of a pixel lives in lanes l, l^1 (next column) and l^Q, l^Q^1
+                                    // (next image row): Q is a power of two <= 16 here, so all four are in this warp
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        f[j] = fmaxf(f[j], __shfl_xor_sync(0xffffffffu, f[j], 1));
+                                        f[j] = fmaxf(f[j], __shfl_xor_sync(0xffffffffu, f[j], p.Q));
+                                    }
+                                    if ((lane & 1) == 0 && (lane & p.Q) == 0) {
+                                        const int prow = (trow / (2 * p.Q)) * (p.Q >> 1) + ((trow & (p.Q - 1)) >> 1);
+                                        *(bf16x8 *)(buf_ptr + sub_off(prow, sb * 2 + h)) = pack8(f);
+                                    }
+                                } else {
+                                    *(bf16x8 *)(buf_ptr + sub_off(trow, sb * 2 + h)) = pack8(f);
+                                }
                             }
                         }
                     }
@@ -543,7 +572,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     ok = epi_sync();
                     if (!ok) break;
                     if (store_thread) {
-                        if (k_base + cg < p.k_pad) tma_store_2d(&tm_y, buf, k_base + cg, (int)m0);
+                        if (k_base + cg < p.k_pad) tma_store_2d(&tm_y, buf, k_base + cg, (int)(POOL ? m0 >> 2 : m0));
                         tma_store_commit();
                     }
                     ++group_counter;
@@ -561,7 +590,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     uint8_t *dst = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 6) * SUB_BYTES + (k & 7) * 2;
                     const uint32_t buf = staging0 + (group_counter & 1u) * GROUP_BYTES;
                     const long long mg = m0 + g * 64;
-                    if (warp_has_work) {
+                    if (warp_has_work && POOL) {
+                        // all 64 pixels of the group for this filter, then the 16 pooled values
+                        uint32_t v[64];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + c * 16), v + c * 16);
+                        tmem_ld_wait();
+                        if (k_ok) {
+                            float f[64];
+#pragma unroll
+                            for (int j = 0; j < 64; ++j) f[j] = apply_act(__uint_as_float(v[j]) + bias, p.act);
+                            uint8_t *pd = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 6) * POOL_SUB_BYTES + (k & 7) * 2;
+                            switch (p.Q) {
+                                case 2: store_pooled<2>(f, pd, hk); break;
+                                case 4: store_pooled<4>(f, pd, hk); break;
+                                case 8: store_pooled<8>(f, pd, hk); break;
+                                case 16: store_pooled<16>(f, pd, hk); break;
+                                default: store_pooled<32>(f, pd, hk); break;
+                            }
+                        }
+                    } else if (warp_has_work) {
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             uint32_t v[32];
@@ -589,8 +637,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     ok = epi_sync();
                     if (!ok) break;
                     if (store_thread) {
-                        for (int sb = 0; sb < n_sub; ++sb)
-                            tma_store_2d(&tm_y, buf + sb * SUB_BYTES, sb * SUB, (int)mg);
+                        for (int sb = 0; sb < n_sub; ++sb) {
+                            if (POOL) tma_store_2d(&tm_y, buf + sb * POOL_SUB_BYTES, sb * SUB, (int)(mg >> 2));
+                            else tma_store_2d(&tm_y, buf + sb * SUB_BYTES, sb * SUB, (int)mg);
+                        }
                         tma_store_commit();
                     }
                     ++group_counter;
@@ -646,33 +696,45 @@ static cprune_status load_driver_entry_points() {
 }
 
 // Split-K finalize: y[m][k] = act(bias[k] + residual[m][k] + sum over slices of partial[s][m][k]),
-// slices added in index order (deterministic).  One thread per (pixel, 8 filters).
+// slices added in index order (deterministic).  One thread per (output pixel, 8 filters).  With
+// pool_q > 0 an output pixel is the maximum over its 2x2 window of conv pixels (image rows of pool_q
+// pixels; a pooled pixel j of an image covers conv pixels 2*(j / (pool_q/2))*pool_q + 2*(j % (pool_q/2)) + {0,1,pool_q,pool_q+1}).
 __global__ void __launch_bounds__(256) splitk_finalize_kernel(const float *__restrict__ partial, int splits, long long M,
                                                               int k_alloc, int k8, const float *__restrict__ bias,
-                                                              const bf16x8 *__restrict__ res, int act,
+                                                              const bf16x8 *__restrict__ res, int act, int pool_q,
                                                               bf16x8 *__restrict__ y) {
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= M * k8) return;
-    const long long m = e / k8;
-    const int kg = (int)(e - m * k8);
-    float f[8];
+    const long long out_pixels = pool_q ? M / 4 : M;
+    if (e >= out_pixels * k8) return;
+    const long long mo = e / k8;
+    const int kg = (int)(e - mo * k8);
+    float bb[8], best[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) f[j] = __ldg(bias + kg * 8 + j);
-    for (int sidx = 0; sidx < splits; ++sidx) {
-        const float4 *src = (const float4 *)(partial + ((size_t)sidx * M + m) * k_alloc + kg * 8);
-        const float4 a = __ldg(src), b = __ldg(src + 1);
-        f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
-        f[4] += b.x; f[5] += b.y; f[6] += b.z; f[7] += b.w;
+    for (int j = 0; j < 8; ++j) { bb[j] = __ldg(bias + kg * 8 + j); best[j] = -INFINITY; }
+    const int windows = pool_q ? 4 : 1;
+    const int hq = pool_q >> 1;
+    for (int wdx = 0; wdx < windows; ++wdx) {
+        long long m = mo;
+        if (pool_q) m = 2 * (mo / hq) * pool_q + 2 * (mo % hq) + (wdx & 1) + (wdx >> 1) * pool_q;
+        float f[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = bb[j];
+        for (int sidx = 0; sidx < splits; ++sidx) {
+            const float4 *src = (const float4 *)(partial + ((size_t)sidx * M + m) * k_alloc + kg * 8);
+            const float4 a = __ldg(src), b = __ldg(src + 1);
+            f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+            f[4] += b.x; f[5] += b.y; f[6] += b.z; f[7] += b.w;
+        }
+        if (res) {
+            float rf[8];
+            unpack8(ldg8(res + m * k8 + kg), rf);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) f[j] += rf[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) best[j] = fmaxf(best[j], apply_act(f[j], act));
     }
-    if (res) {
-        float rf[8];
-        unpack8(ldg8(res + e), rf);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) f[j] += rf[j];
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], act);
-    y[e] = pack8(f);
+    y[e] = pack8(best);
 }
 
 // 128 x 128 identity in bf16: the filter-side operand of the residual blocks (see the producer).
@@ -799,6 +861,15 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
         int sp = atoi(force);
         if (sp >= 1 && !plan->small_c && sp <= iters && (sp - 1) * ((iters + sp - 1) / sp) < iters) plan->splits = sp;
     }
+    // A 2x2 max-pool is fused when a tile holds whole pairs of image rows: Q a power of two with the
+    // four pixels of a window in one warp (pixel-major: Q <= 16) or in one thread's 64-pixel group
+    // (filter-major: Q <= 32).  The split-K finalize kernel pools for any even P, Q.
+    plan->fused_pool = 0;
+    if (plan->opts.pool == CPRUNE_POOL_MAX2X2) {
+        const bool pow2 = (i.Q & (i.Q - 1)) == 0 && i.Q >= 2;
+        if (plan->splits > 1) plan->fused_pool = 1;
+        else if (pow2 && i.Q <= (plan->orient == ORIENT_PIX ? 16 : 32)) plan->fused_pool = 1;
+    }
     plan->ipp = (iters + plan->splits - 1) / plan->splits;
     plan->partial_bytes = plan->splits > 1 ? (size_t)plan->splits * (size_t)M * i.k_alloc * 4 : 0;
     return CPRUNE_OK;
@@ -843,10 +914,11 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
     }
     if (plan->map_y != y) {
         // output as a 2-D tensor [pixels][k_pad]; stored in boxes of 64 filters x 128 or 64 pixels
-        const long long M = (long long)i.N * i.P * i.Q;
+        // (with a fused 2x2 pool: [pooled pixels][k_pad], boxes of 32 or 16 pooled pixels)
+        const long long M = (long long)i.N * i.P * i.Q / (plan->fused_pool ? 4 : 1);
         cuuint64_t dims[2] = {(cuuint64_t)i.k_pad, (cuuint64_t)M};
         cuuint64_t strides[1] = {(cuuint64_t)i.k_pad * 2};
-        cuuint32_t box[2] = {SUB, (cuuint32_t)(plan->orient == ORIENT_PIX ? 128 : 64)};
+        cuuint32_t box[2] = {SUB, (cuuint32_t)((plan->orient == ORIENT_PIX ? 128 : 64) / (plan->fused_pool ? 4 : 1))};
         cuuint32_t estr[2] = {1, 1};
         CUresult r = g_encode_tiled(&plan->tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -915,8 +987,10 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     {
         std::lock_guard<std::mutex> lock(attr_mu);
         if (!attr_set) {
-            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_PIX>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_FILT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_PIX, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_PIX, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_FILT, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_FILT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             attr_set = 1;
         }
     }
@@ -928,6 +1002,7 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     p.PT = i.tile_m; p.FT = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
     p.small_c = plan->small_c;
     p.splits = plan->splits;
+    p.pool = plan->fused_pool;
     p.ipp = plan->ipp;
     p.k_alloc = i.k_alloc;
     p.partial = (float *)partial;
@@ -942,16 +1017,21 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     const int total = i.tiles_m * i.tiles_n * plan->splits;
     if (total == 0) return CPRUNE_OK;
     const int grid = total < sm_count() ? total : sm_count();
-    if (plan->orient == ORIENT_PIX)
-        conv_tc_kernel<ORIENT_PIX><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
-    else
-        conv_tc_kernel<ORIENT_FILT><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+    const bool pool_in_kernel = plan->fused_pool && !split;
+    if (plan->orient == ORIENT_PIX) {
+        if (pool_in_kernel) conv_tc_kernel<ORIENT_PIX, 1><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+        else conv_tc_kernel<ORIENT_PIX, 0><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+    } else {
+        if (pool_in_kernel) conv_tc_kernel<ORIENT_FILT, 1><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+        else conv_tc_kernel<ORIENT_FILT, 0><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+    }
     CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
     if (split) {
-        const long long elems = p.M * (i.k_pad / 8);
+        const long long elems = (plan->fused_pool ? p.M / 4 : p.M) * (i.k_pad / 8);
         splitk_finalize_kernel<<<(unsigned)ceil_div(elems, 256), 256, 0, st>>>((const float *)partial, plan->splits, p.M,
                                                                               i.k_alloc, i.k_pad / 8, b, (const bf16x8 *)res,
-                                                                              plan->opts.activation, (bf16x8 *)y);
+                                                                              plan->opts.activation,
+                                                                              plan->fused_pool ? i.Q : 0, (bf16x8 *)y);
         CPRUNE_LAUNCH_CHECK("splitk_finalize_kernel");
     }
     return CPRUNE_OK;

@@ -122,7 +122,7 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
                 }
                 o.h = i.out_h; o.w = i.out_w; o.c = i.K;
                 if (i.workspace_bytes > m->workspace_bytes) m->workspace_bytes = i.workspace_bytes;
-                m->launches += (d.plan->opts.pool ? 2 : 1) + (d.plan->splits > 1 ? 1 : 0);
+                m->launches += ((d.plan->opts.pool && !(i.kernel == CPRUNE_KERNEL_TENSOR && d.plan->fused_pool)) ? 2 : 1) + (d.plan->splits > 1 ? 1 : 0);
                 break;
             }
             case CPRUNE_OP_MAXPOOL:

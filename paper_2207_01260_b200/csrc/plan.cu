@@ -72,7 +72,8 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * i.S * i.c_pad * 2;
     i.packed_bias_bytes = (size_t)i.k_alloc * sizeof(float);
     // workspace: [unpooled conv output if a pool follows][split-K partial sums]
-    pl->pool_bytes = pl->opts.pool == CPRUNE_POOL_MAX2X2 ? ((size_t)i.N * i.P * i.Q * i.k_pad * 2 + 255) / 256 * 256 : 0;
+    const bool separate_pool = pl->opts.pool == CPRUNE_POOL_MAX2X2 && !(family == CPRUNE_KERNEL_TENSOR && pl->fused_pool);
+    pl->pool_bytes = separate_pool ? ((size_t)i.N * i.P * i.Q * i.k_pad * 2 + 255) / 256 * 256 : 0;
     i.workspace_bytes = pl->pool_bytes + (family == CPRUNE_KERNEL_TENSOR ? pl->partial_bytes : 0);
     i.algorithmic_bytes = 2.0 * ((double)i.N * i.H * i.W * i.C + (double)i.N * i.out_h * i.out_w * i.K +
                                  (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
@@ -170,7 +171,7 @@ cprune_status cprune_task_run(cprune_plan *plan, const void *x, const void *w_pa
     if (((uintptr_t)x | (uintptr_t)w_packed | (uintptr_t)y | (uintptr_t)residual | (uintptr_t)workspace) & 15)
         return CPRUNE_ERR_INVALID_ARG;
     const cprune_plan_info &i = plan->info;
-    const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
+    const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2 && !(i.kernel == CPRUNE_KERNEL_TENSOR && plan->fused_pool);
     if (i.workspace_bytes && !workspace) return CPRUNE_ERR_INVALID_ARG;
     void *conv_out = pool ? workspace : y;
     void *partial = plan->partial_bytes ? (void *)((char *)workspace + plan->pool_bytes) : nullptr;

@@ -28,6 +28,7 @@ struct cprune_plan {
     int smem_bytes = 0;
     int orient = 0;                 // which side of the MMA the pixels are on
     int staging_bufs = 2;
+    int fused_pool = 0;             // the 2x2 max-pool runs inside the conv kernel / the split-K finalize kernel
     int splits = 1;                 // split-K slices per output tile
     int ipp = 0;                    // K blocks per slice
     size_t pool_bytes = 0;          // unpooled conv output in the workspace when a 2x2 pool follows

@@ -157,6 +157,16 @@ def test_dense_task_epilogues(cp, kernel):
     check_task(cp, 1, 64, 8, 8, 64, 3, 1, 1, act="none", kernel=kernel)
 
 
+@pytest.mark.parametrize("case", [
+    # N, C, HW, K: fused in the filter-major epilogue (Q = 32, 16, 4), in the pixel-major epilogue (Q = 8, 2),
+    # in the split-K finalize kernel (few tiles), and as a separate pass (Q not a power of two)
+    (3, 45, 32, 58), (2, 101, 16, 96), (5, 20, 4, 40), (4, 171, 8, 163), (40, 64, 2, 243), (2, 250, 4, 212),
+    (1, 24, 12, 32), (1, 200, 12, 200)])
+def test_fused_maxpool(cp, case):
+    N, C, HW, K = case
+    check_task(cp, N, C, HW, HW, K, 3, 1, 1, act="relu", pool="max2x2", kernel="tensor")
+
+
 @pytest.mark.parametrize("C", [64, 65, 66, 67, 68, 69, 70, 71, 72, 73, 79, 80, 81])
 def test_every_channel_residue(cp, C):
     # C and K sweep the residues modulo 8 and 16 around a 64-channel block boundary
