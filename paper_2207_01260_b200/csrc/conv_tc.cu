@@ -54,18 +54,22 @@ struct TcParams {
     int ksteps_last;   // 16-channel MMA steps in the last channel block
     int PT, FT;        // pixels and filters per tile
     int tiles_m, tiles_n, k_pad, stages, act;
-    int small_c;       // c_pad == 8 (3-channel stems): a 64-wide K block is 8 taps x 8 channels
+    int small_c;       // c_pad == 8 (3-channel stems): 1 = a 64-wide K block is 8 taps x 8 channels;
+                       // 2 = stride-2 stems read as pixel pairs: 4 pair-taps x 16 channels per K block
+    int pair_taps;     // small_c == 2: pair-taps per filter row, (S + 1) / 2
     int iters;         // pipeline stages per tile (K blocks, plus residual blocks)
     int res_iters;     // ORIENT_FILT with a residual: trailing stages that add it on the tensor core
     int pool;          // 1: 2x2 stride-2 max-pool fused into the epilogue (tm_y then maps the pooled output)
     int splits;        // split-K: CTAs that share one output tile, each a slice of the K blocks
     int ipp;           // K blocks per slice
-    int k_alloc;       // row length of the float32 partial sums
     float *partial;    // [splits][M][k_alloc] when splits > 1
     const float *bias;
     const __nv_bfloat16 *res;
     int *status;
 };
+// Measured on B200: with kernel parameters beyond 768 bytes (five 128-byte tensor maps + this struct) tasks with
+// many short tiles ran almost twice as slow; the struct therefore has to stay within 128 bytes.
+static_assert(sizeof(TcParams) <= 128, "conv_tc_kernel parameters must stay within 768 bytes");
 
 // ------------------------------------------------------------------------------------------ PTX
 
@@ -220,6 +224,18 @@ __device__ __forceinline__ uint64_t smem_desc_interleaved(uint32_t addr, uint32_
     return d;
 }
 
+// Descriptor of a K-major bf16 operand whose rows are 32 bytes (16 channels), 32-byte swizzled, 8-row groups
+// 256 bytes apart: one im2col load of 16 channels per (paired) pixel = exactly one K = 16 step.
+__device__ __forceinline__ uint64_t smem_desc_sw32(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(256 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;                  // 32-byte swizzle
+    return d;
+}
+
 // Byte offset of (row, 16-byte chunk c of 8) in a staged sub-tile of 128-byte rows under the
 // 128-byte swizzle (address bits 4..6 are XORed with bits 7..9, i.e. with the row modulo 8).
 __device__ __forceinline__ uint32_t sub_off(int row, int c) { return (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)); }
@@ -291,6 +307,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    const int k_alloc = p.tiles_n * p.FT;     // row length of the float32 partial sums (split-K)
     const int total_tiles = p.tiles_m * p.tiles_n * p.splits;   // work items: (tile, K slice), slice fastest
     const int PQ = p.P * p.Q;
 
@@ -308,7 +325,31 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             const int rem = (int)(m0 - (long long)n_img * PQ);
             const int p0 = rem / p.Q, q0 = rem - p0 * p.Q;
             const int wc = q0 * p.stride - p.pad, hc = p0 * p.stride - p.pad;
-            if (p.small_c) {
+            if (p.small_c == 2) {
+                // stride-2 stem read as pixel pairs: the tensor map sees [N][H][W/2][16]; a pair-tap is one im2col
+                // load of PT pixels x 32 bytes = one K step; 4 pair-taps per stage
+                const int taps = p.R * p.pair_taps;
+                const int wcp = q0 - ((p.pad + 1) >> 1);
+                for (int it = 0; it < p.iters - p.res_iters; ++it) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                    if (!ok) break;
+                    if (elect_one()) {
+                        const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
+                        int loads = taps - it * 4;
+                        if (loads > 4) loads = 4;
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(loads * p.PT * 32 + p.FT * BK * 2));
+                        for (int t = 0; t < loads; ++t) {
+                            const int tap = it * 4 + t;
+                            const int r = tap / p.pair_taps, tp = tap - r * p.pair_taps;
+                            tma_load_im2col(x_dst + (uint32_t)(t * p.PT * 32), &tm_x, full_bar(stage), 0, wcp, hc, n_img,
+                                            (uint16_t)tp, (uint16_t)r);
+                        }
+                        tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), it * BK, 0, nt_f * p.FT);
+                    }
+                    __syncwarp();
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            } else if (p.small_c) {
                 // 8 taps x 8 channels per stage; every tap is its own im2col load of PT pixels x 16 bytes
                 const int taps = p.R * p.S;
                 for (int it = 0; it < p.iters - p.res_iters; ++it) {
@@ -392,6 +433,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     int left = p.k_pad - (it - main_iters) * BK;
                     if (left > BK) left = BK;
                     nk = (left + 15) >> 4;
+                } else if (p.small_c == 2) {
+                    nk = p.R * p.pair_taps - it * 4;
+                    if (nk > 4) nk = 4;
                 } else if (p.small_c) {
                     int nt = p.R * p.S - it * 8;
                     if (nt > 8) nt = 8;
@@ -400,7 +444,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     nk = ((it + 1) % p.cblks == 0) ? p.ksteps_last : BK / 16;
                 }
                 if (elect_one()) {
-                    if (p.small_c && !res_it) {
+                    if (p.small_c == 2 && !res_it) {
+                        // pixel operand: one pair-tap (16 channels) per MMA, pair-taps PT*32 bytes apart
+                        for (int kk = 0; kk < nk; ++kk) {
+                            const uint64_t dxp = smem_desc_sw32(x_addr + (uint32_t)kk * (uint32_t)p.PT * 32u);
+                            if (ORIENT == ORIENT_PIX)
+                                umma_bf16(d_tmem, dxp, dw + (uint64_t)(2 * kk), idesc, accumulate);
+                            else
+                                umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dxp, idesc, accumulate);
+                            accumulate = 1;
+                        }
+                    } else if (p.small_c && !res_it) {
                         // pixel operand: two taps (2 x 8 channels) per MMA, taps PT*16 bytes apart
                         const uint32_t tap_bytes = (uint32_t)p.PT * 16u;
                         for (int kk = 0; kk < nk; ++kk) {
@@ -468,7 +522,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             if (p.splits > 1) {
                 // split-K: this CTA holds a partial sum; store it as float32, the finalize kernel adds
                 // the slices in a fixed order and applies bias, residual and activation
-                float *part = p.partial + (size_t)split * (size_t)p.M * p.k_alloc;
+                float *part = p.partial + (size_t)split * (size_t)p.M * k_alloc;
                 if (ORIENT == ORIENT_PIX) {
                     const long long m = m0 + trow;
                     for (int c0 = 0; c0 < p.FT; c0 += 16) {
@@ -476,7 +530,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                         tmem_ld16(t_row + (uint32_t)c0, v);
                         tmem_ld_wait();
                         if (m < p.M) {
-                            float4 *dst = (float4 *)(part + (size_t)m * p.k_alloc + k_base + c0);
+                            float4 *dst = (float4 *)(part + (size_t)m * k_alloc + k_base + c0);
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
                                 dst[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
@@ -493,7 +547,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const long long m = m0 + c0 + j;
-                                if (m < p.M) part[(size_t)m * p.k_alloc + k] = __uint_as_float(v[j]);
+                                if (m < p.M) part[(size_t)m * k_alloc + k] = __uint_as_float(v[j]);
                             }
                         }
                     }
@@ -797,6 +851,13 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     const int k16 = round_up(i.K, 16);
     int PT, FT, tiles_n, bufs, group_rows;
     plan->small_c = (i.c_pad == 8 && i.K <= 128 && i.R * i.S > 1) ? 1 : 0;
+    // stride-2 stems with odd pad and odd S: read the image as pixel pairs (16 channels per pair), which halves
+    // the number of loads and doubles their row width; the packed filters get one zero tap in front of each row
+    if (plan->small_c && i.stride == 2 && (i.W & 1) == 0 && (i.pad & 1) == 1 && (i.S & 1) == 1) plan->small_c = 2;
+    if (const char *e = getenv("CPRUNE_STEM_PAIRS")) {      // measurement override
+        if (e[0] == '0' && plan->small_c == 2) plan->small_c = 1;
+    }
+    plan->s_packed = plan->small_c == 2 ? i.S + 1 : i.S;
     if (i.K <= 128) {
         // filters on the MMA-M side (padded to 128 rows), 256 pixels on the MMA-N side
         plan->orient = ORIENT_FILT;
@@ -832,7 +893,8 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     const int cblks = (i.c_pad + BK - 1) / BK;
     const int ksteps = (cblks - 1) * (BK / 16) + (i.c_pad - (cblks - 1) * BK + 15) / 16;
     i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * (double)(i.R * i.S) * ksteps * 16.0;
-    if (plan->small_c) i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * ((i.R * i.S + 1) / 2) * 16.0;
+    if (plan->small_c == 1) i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * ((i.R * i.S + 1) / 2) * 16.0;
+    if (plan->small_c == 2) i.padded_flops = 2.0 * (double)i.tiles_m * PT * (double)i.k_alloc * (i.R * (i.S + 1) / 2) * 16.0;
     plan->staging_bufs = bufs;
     plan->smem_bytes = smem_for(stages, PT, FT, bufs, group_rows);
     // Split-K when the tiles cannot fill the SMs: slices of the K blocks go to different CTAs, which
@@ -886,11 +948,22 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         int lower[2] = {-i.pad, -i.pad};
         int upper[2] = {i.pad - (i.S - 1), i.pad - (i.R - 1)};
         cuuint32_t estr[4] = {1, (cuuint32_t)i.stride, (cuuint32_t)i.stride, 1};
-        // small-C mode: 8 channels (16 bytes) per pixel, dense rows, no swizzle
+        cuuint32_t chans = BK;
+        CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B;
+        if (plan->small_c == 1) {          // 8 channels (16 bytes) per pixel, dense rows, no swizzle
+            chans = 8;
+            swz = CU_TENSOR_MAP_SWIZZLE_NONE;
+        } else if (plan->small_c == 2) {   // the same memory seen as [N][H][W/2][16]: pixel pairs, unit step along W/2
+            dims[0] = 16; dims[1] = (cuuint64_t)i.W / 2;
+            strides[0] = 32;
+            lower[0] = -((i.pad + 1) / 2);
+            upper[0] = i.Q - i.W / 2 + lower[0];   // exactly Q start positions per image row
+            estr[1] = 1;
+            chans = 16;
+            swz = CU_TENSOR_MAP_SWIZZLE_32B;
+        }
         CUresult r = g_encode_im2col(&plan->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), dims, strides,
-                                     lower, upper, plan->small_c ? 8 : BK, (cuuint32_t)i.tile_m, estr,
-                                     CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                     plan->small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                                     lower, upper, chans, (cuuint32_t)i.tile_m, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeIm2col");
         // Drivers up to 13.1 set a descriptor bit for im2col maps of tensors smaller than 128 KiB
@@ -900,10 +973,11 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
         plan->map_x = x;
     }
     if (plan->map_w != w) {
-        // small-C mode reads a filter row [R*S taps][8 channels] as one long channel axis
-        cuuint64_t dims[3] = {(cuuint64_t)(plan->small_c ? i.R * i.S * 8 : i.c_pad), (cuuint64_t)(plan->small_c ? 1 : i.R * i.S),
+        // small-C modes read a filter row [R * s_packed taps][8 channels] as one long channel axis
+        const int row_elems = i.R * plan->s_packed * i.c_pad;
+        cuuint64_t dims[3] = {(cuuint64_t)(plan->small_c ? row_elems : i.c_pad), (cuuint64_t)(plan->small_c ? 1 : i.R * i.S),
                               (cuuint64_t)i.k_alloc};
-        cuuint64_t strides[2] = {(cuuint64_t)(plan->small_c ? i.R * i.S * 8 : i.c_pad) * 2, (cuuint64_t)i.R * i.S * i.c_pad * 2};
+        cuuint64_t strides[2] = {(cuuint64_t)(plan->small_c ? row_elems : i.c_pad) * 2, (cuuint64_t)row_elems * 2};
         cuuint32_t box[3] = {BK, 1, (cuuint32_t)i.tile_n};
         cuuint32_t estr[3] = {1, 1, 1};
         CUresult r = g_encode_tiled(&plan->tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w), dims, strides, box,
@@ -1001,13 +1075,15 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     p.ksteps_last = (i.c_pad - (p.cblks - 1) * BK + 15) / 16;
     p.PT = i.tile_m; p.FT = i.tile_n; p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.k_pad = i.k_pad; p.stages = i.stages;
     p.small_c = plan->small_c;
+    p.pair_taps = (i.S + 1) / 2;
     p.splits = plan->splits;
     p.pool = plan->fused_pool;
     p.ipp = plan->ipp;
-    p.k_alloc = i.k_alloc;
     p.partial = (float *)partial;
     p.res_iters = mma_res ? (i.k_pad + BK - 1) / BK : 0;
-    p.iters = (plan->small_c ? (i.R * i.S + 7) / 8 : i.R * i.S * p.cblks) + p.res_iters;
+    const int main_iters = plan->small_c == 2 ? (i.R * p.pair_taps + 3) / 4
+                           : plan->small_c == 1 ? (i.R * i.S + 7) / 8 : i.R * i.S * p.cblks;
+    p.iters = main_iters + p.res_iters;
     if (plan->splits == 1) p.ipp = p.iters;   // one slice covers everything, the residual blocks included
     p.act = plan->opts.activation;
     p.bias = b;

@@ -5,18 +5,19 @@
 
 namespace cprune {
 
-// dense: out[k][r][s][c] for k < k_alloc, c < c_pad; zero where k >= K or c >= C
-__global__ void pack_dense_kernel(const float *__restrict__ w, int K, int C, int R, int S, int k_alloc, int c_pad,
-                                  __nv_bfloat16 *__restrict__ out) {
-    size_t total = (size_t)k_alloc * R * S * c_pad;
+// dense: out[k][r][s'][c] for k < k_alloc, s' < S_out, c < c_pad, where tap s' holds filter tap s = s' - s_off
+// (s_off = 1 puts one zero tap in front of every filter row); zero where k >= K, c >= C or s is out of range
+__global__ void pack_dense_kernel(const float *__restrict__ w, int K, int C, int R, int S, int S_out, int s_off, int k_alloc,
+                                  int c_pad, __nv_bfloat16 *__restrict__ out) {
+    size_t total = (size_t)k_alloc * R * S_out * c_pad;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
         int c = (int)(e % c_pad);
         size_t t = e / c_pad;
-        int s = (int)(t % S);
-        t /= S;
+        int s = (int)(t % S_out) - s_off;
+        t /= S_out;
         int r = (int)(t % R);
         int k = (int)(t / R);
-        float v = (k < K && c < C) ? w[(((size_t)k * C + c) * R + r) * S + s] : 0.f;
+        float v = (k < K && c < C && s >= 0 && s < S) ? w[(((size_t)k * C + c) * R + r) * S + s] : 0.f;
         out[e] = __float2bfloat16_rn(v);
     }
 }
@@ -67,10 +68,11 @@ static int grid_for(size_t total, int threads) {
     return (int)g;
 }
 
-cprune_status pack_dense(const float *w, const float *b, int K, int C, int R, int S, int k_alloc, int c_pad,
+cprune_status pack_dense(const float *w, const float *b, int K, int C, int R, int S, int S_out, int k_alloc, int c_pad,
                          void *w_packed, float *b_packed, cudaStream_t st) {
-    size_t total = (size_t)k_alloc * R * S * c_pad;
-    pack_dense_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, K, C, R, S, k_alloc, c_pad, (__nv_bfloat16 *)w_packed);
+    size_t total = (size_t)k_alloc * R * S_out * c_pad;
+    pack_dense_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, K, C, R, S, S_out, S_out - S, k_alloc, c_pad,
+                                                           (__nv_bfloat16 *)w_packed);
     CPRUNE_LAUNCH_CHECK("pack_dense_kernel");
     pad_bias_kernel<<<(k_alloc + 255) / 256, 256, 0, st>>>(b, K, k_alloc, b_packed);
     CPRUNE_LAUNCH_CHECK("pad_bias_kernel");
@@ -96,13 +98,14 @@ cprune_status cprune_pack_weights(const cprune_plan *plan, const float *w, const
         CPRUNE_LAUNCH_CHECK("pad_bias_kernel");
         return CPRUNE_OK;
     }
-    return pack_dense(w, b, i.K, i.C, i.R, i.S, i.k_alloc, i.c_pad, w_packed, b_packed, st);
+    const int s_out = (i.kernel == CPRUNE_KERNEL_TENSOR && plan->s_packed > 0) ? plan->s_packed : i.S;
+    return pack_dense(w, b, i.K, i.C, i.R, i.S, s_out, i.k_alloc, i.c_pad, w_packed, b_packed, st);
 }
 
 cprune_status cprune_fc_pack(const float *w, const float *b, int out, int in, void *w_packed, float *b_packed,
                              void *stream) {
     if (!w || !w_packed || !b_packed || out <= 0 || in <= 0) return CPRUNE_ERR_INVALID_ARG;
-    return pack_dense(w, b, out, in, 1, 1, cprune_padded_channels(out), cprune_padded_channels(in), w_packed, b_packed,
+    return pack_dense(w, b, out, in, 1, 1, 1, cprune_padded_channels(out), cprune_padded_channels(in), w_packed, b_packed,
                       (cudaStream_t)stream);
 }
 

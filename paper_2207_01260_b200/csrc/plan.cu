@@ -69,7 +69,8 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     if (st != CPRUNE_OK) { delete pl; return st; }
     i.kernel = family;
     const double rs = (double)i.R * i.S;
-    i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * i.S * i.c_pad * 2;
+    const int s_packed = (family == CPRUNE_KERNEL_TENSOR && pl->s_packed > 0) ? pl->s_packed : i.S;
+    i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * s_packed * i.c_pad * 2;
     i.packed_bias_bytes = (size_t)i.k_alloc * sizeof(float);
     // workspace: [unpooled conv output if a pool follows][split-K partial sums]
     const bool separate_pool = pl->opts.pool == CPRUNE_POOL_MAX2X2 && !(family == CPRUNE_KERNEL_TENSOR && pl->fused_pool);

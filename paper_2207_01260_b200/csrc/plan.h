@@ -33,7 +33,8 @@ struct cprune_plan {
     int ipp = 0;                    // K blocks per slice
     size_t pool_bytes = 0;          // unpooled conv output in the workspace when a 2x2 pool follows
     size_t partial_bytes = 0;       // float32 partial sums in the workspace
-    int small_c = 0;                // 3-channel stems: 8 taps x 8 channels per K block
+    int small_c = 0;                // 3-channel stems: 1 = 8 taps x 8 channels per K block, 2 = pixel pairs
+    int s_packed = 0;               // filter taps per row in the packed weights (S, or S + 1 in pair mode)
 };
 
 namespace cprune {
