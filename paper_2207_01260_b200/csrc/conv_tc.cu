@@ -858,7 +858,12 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
         if (e[0] == '0' && plan->small_c == 2) plan->small_c = 1;
     }
     plan->s_packed = plan->small_c == 2 ? i.S + 1 : i.S;
-    if (i.K <= 128) {
+    // Orientation.  K <= 128: filters on the 128-row side (256 pixels per MMA) -- except for tasks with one or two
+    // K blocks and at most 32 filters (MobileNetV2 project layers), where the pixel-major epilogue, in which every
+    // thread stores one pixel's contiguous filters, is faster than the transposing one (measured: 45 vs 62 us).
+    const int k_blocks = i.R * i.S * ((i.c_pad + BK - 1) / BK);
+    const bool few_filters = !plan->small_c && k_blocks <= 2 && i.K <= 32;
+    if (i.K <= 128 && !few_filters) {
         // filters on the MMA-M side (padded to 128 rows), 256 pixels on the MMA-N side
         plan->orient = ORIENT_FILT;
         PT = 256; FT = 128; tiles_n = 1; bufs = 2; group_rows = 64;
