@@ -496,6 +496,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         uint32_t acc_phase = 0, epi_phase = 0;
         uint32_t group_counter = 0;                    // staged groups so far (selects the buffer)
         bool ok = true;
+        // filter-major orientation: this thread's filter and its bias are the same for every tile
+        const float filt_bias = (ORIENT == ORIENT_FILT && trow < p.k_pad) ? __ldg(p.bias + trow) : 0.f;
         // Bounded barrier among the four epilogue warps (one arrival per warp).  Per staged group:
         // everyone writes buffer g%2, the store thread makes sure every earlier store has been read
         // out of shared memory, all meet here, then the store thread issues the stores of group g.
@@ -635,7 +637,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 // rows = filters, columns = pixels; groups of 64 pixels
                 const int k = trow;                       // this thread's filter
                 const bool k_ok = k < p.k_pad;
-                const float bias = k_ok ? __ldg(p.bias + k) : 0.f;
+                const float bias = filt_bias;
                 const int n_sub = (p.k_pad + SUB - 1) / SUB;       // sub-tiles that hold real filters
                 const bool warp_has_work = quarter * 32 < p.k_pad; // all 32 filters of this warp may be padding
                 const int groups = p.PT / 64;
@@ -664,20 +666,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                             }
                         }
                     } else if (warp_has_work) {
+                        uint32_t v[64];
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            uint32_t v[32];
-                            tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32), v);
-                            tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32 + 16), v + 16);
-                            tmem_ld_wait();
-                            if (k_ok) {
+                        for (int c = 0; c < 4; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + c * 16), v + c * 16);
+                        tmem_ld_wait();
+                        if (k_ok) {
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const int px = half * 32 + j;
-                                    float f = __uint_as_float(v[j]) + bias;
-                                    f = apply_act(f, p.act);
-                                    *(__nv_bfloat16 *)(dst + sub_off(px, hk)) = __float2bfloat16_rn(f);
-                                }
+                            for (int px = 0; px < 64; ++px) {
+                                float f = __uint_as_float(v[px]) + bias;
+                                f = apply_act(f, p.act);
+                                *(__nv_bfloat16 *)(dst + sub_off(px, hk)) = __float2bfloat16_rn(f);
                             }
                         }
                     }
