@@ -35,7 +35,7 @@
 
 namespace cprune {
 
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;    // producer warp, MMA warp, eight epilogue warps
 constexpr int BK = 64;             // channels per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;    // column offset of the second accumulator buffer
@@ -240,16 +240,16 @@ __device__ __forceinline__ uint64_t smem_desc_sw32(uint32_t addr) {
 // 128-byte swizzle (address bits 4..6 are XORed with bits 7..9, i.e. with the row modulo 8).
 __device__ __forceinline__ uint32_t sub_off(int row, int c) { return (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)); }
 
-// 2x2 stride-2 max-pool of 64 consecutive pixels (rows of Q pixels, Q a power of two <= 32) held by one
-// thread for one filter: 16 pooled values, written to rows 0..15 of a staged sub-tile.
-template <int Q>
-__device__ __forceinline__ void store_pooled(const float *f, uint8_t *dst, int chunk) {
+// 2x2 stride-2 max-pool of NPX consecutive pixels (whole row pairs of Q pixels, Q a power of two) held by
+// one thread for one filter: NPX / 4 pooled values, written to rows t0.. of a staged sub-tile.
+template <int Q, int NPX>
+__device__ __forceinline__ void store_pooled(const float *f, uint8_t *dst, int chunk, int t0) {
 #pragma unroll
-    for (int t = 0; t < 16; ++t) {
+    for (int t = 0; t < NPX / 4; ++t) {
         const int rp = t / (Q / 2), cq = t % (Q / 2);
         const int b = rp * 2 * Q + 2 * cq;
         const float m = fmaxf(fmaxf(f[b], f[b + 1]), fmaxf(f[b + Q], f[b + Q + 1]));
-        *(__nv_bfloat16 *)(dst + sub_off(t, chunk)) = __float2bfloat16_rn(m);
+        *(__nv_bfloat16 *)(dst + sub_off(t0 + t, chunk)) = __float2bfloat16_rn(m);
     }
 }
 
@@ -292,9 +292,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 4);
+            mbar_init(tempty_bar(a), 8);
         }
-        mbar_init(epi_bar, 4);
+        mbar_init(epi_bar, 8);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -488,17 +488,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ epilogue
-        const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-        const int et = (warp - 2) * 32 + lane;         // 0..127 among the epilogue threads
+        // Two warps share each quarter of the tensor-memory lanes (a warp may only read lanes 32*(warp%4)..+31):
+        // `half` says which half of every group's columns this warp takes.
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int trow = quarter * 32 + lane;          // accumulator row (pixel or filter) of this thread
-        const bool store_thread = et == 0;
+        const bool store_thread = warp == 2 && lane == 0;
         int acc = 0;
         uint32_t acc_phase = 0, epi_phase = 0;
         uint32_t group_counter = 0;                    // staged groups so far (selects the buffer)
         bool ok = true;
         // filter-major orientation: this thread's filter and its bias are the same for every tile
         const float filt_bias = (ORIENT == ORIENT_FILT && trow < p.k_pad) ? __ldg(p.bias + trow) : 0.f;
-        // Bounded barrier among the four epilogue warps (one arrival per warp).  Per staged group:
+        // Bounded barrier among the eight epilogue warps (one arrival per warp).  Per staged group:
         // everyone writes buffer g%2, the store thread makes sure every earlier store has been read
         // out of shared memory, all meet here, then the store thread issues the stores of group g.
         // Buffer g%2 was last used by group g-2, whose store was confirmed read before barrier g-1.
@@ -514,7 +516,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
             const long long m0 = (long long)mt * p.PT;
             const int k_base = nt * p.FT;
-            // the epilogue ignores the abort flag: all four warps must take the same decisions,
+            // the epilogue ignores the abort flag: all eight warps must take the same decisions,
             // and they all watch the same barriers
             ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, false));
             if (!ok) break;
@@ -527,7 +529,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 float *part = p.partial + (size_t)split * (size_t)p.M * k_alloc;
                 if (ORIENT == ORIENT_PIX) {
                     const long long m = m0 + trow;
-                    for (int c0 = 0; c0 < p.FT; c0 += 16) {
+                    for (int c0 = half * 16; c0 < p.FT; c0 += 32) {
                         uint32_t v[16];
                         tmem_ld16(t_row + (uint32_t)c0, v);
                         tmem_ld_wait();
@@ -542,7 +544,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 } else {
                     const int k = trow;
                     if (quarter * 32 < p.k_pad) {
-                        for (int c0 = 0; c0 < p.PT; c0 += 16) {
+                        for (int c0 = half * 16; c0 < p.PT; c0 += 32) {
                             uint32_t v[16];
                             tmem_ld16(t_row + (uint32_t)c0, v);
                             tmem_ld_wait();
@@ -567,18 +569,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     uint8_t *buf_ptr = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES;
                     const uint32_t buf = staging0 + (group_counter & 1u) * GROUP_BYTES;
                     const int cg = g * 64;                       // first filter column of the group
-                    // residual of this group: 64 filters = 128 contiguous bytes of the thread's row
-                    bf16x8 rv[8];
+                    // this warp's half of the group: 32 filters = 64 contiguous bytes of the thread's row
+                    const int ch = cg + half * 32;
+                    bf16x8 rv[4];
                     if (has_res) {
-                        const __nv_bfloat16 *rrow = p.res + (size_t)m * p.k_pad + k_base + cg;
+                        const __nv_bfloat16 *rrow = p.res + (size_t)m * p.k_pad + k_base + ch;
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (k_base + cg + j * 8 < p.k_pad) rv[j] = ldg8((const bf16x8 *)(rrow + j * 8));
+                        for (int j = 0; j < 4; ++j)
+                            if (k_base + ch + j * 8 < p.k_pad) rv[j] = ldg8((const bf16x8 *)(rrow + j * 8));
                     }
-                    uint32_t v[64];
+                    uint32_t v[32];
 #pragma unroll
-                    for (int sb = 0; sb < 4; ++sb)
-                        if (cg + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(cg + sb * 16), v + sb * 16);
+                    for (int sb = 0; sb < 2; ++sb)
+                        if (ch + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(ch + sb * 16), v + sb * 16);
                     tmem_ld_wait();
                     if (g == groups - 1) {               // accumulator fully read: hand it back to the MMA warp
                         tc_fence_before();
@@ -586,8 +589,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                         if (lane == 0) mbar_arrive(tempty_bar(acc));
                     }
 #pragma unroll
-                    for (int sb = 0; sb < 4; ++sb) {
-                        const int c0 = cg + sb * 16;
+                    for (int sb = 0; sb < 2; ++sb) {
+                        const int c0 = ch + sb * 16;
                         if (c0 < p.FT) {
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
@@ -605,6 +608,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                 }
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], p.act);
+                                const int chunk = half * 4 + sb * 2 + h;      // 16-byte chunk within the 128-byte staged row
                                 if (POOL) {
                                     // the 2x2 window of a pixel lives in lanes l, l^1 (next column) and l^Q, l^Q^1
                                     // (next image row): Q is a power of two <= 16 here, so all four are in this warp
@@ -615,10 +619,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                                     }
                                     if ((lane & 1) == 0 && (lane & p.Q) == 0) {
                                         const int prow = (trow / (2 * p.Q)) * (p.Q >> 1) + ((trow & (p.Q - 1)) >> 1);
-                                        *(bf16x8 *)(buf_ptr + sub_off(prow, sb * 2 + h)) = pack8(f);
+                                        *(bf16x8 *)(buf_ptr + sub_off(prow, chunk)) = pack8(f);
                                     }
                                 } else {
-                                    *(bf16x8 *)(buf_ptr + sub_off(trow, sb * 2 + h)) = pack8(f);
+                                    *(bf16x8 *)(buf_ptr + sub_off(trow, chunk)) = pack8(f);
                                 }
                             }
                         }
@@ -646,36 +650,50 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     uint8_t *dst = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 6) * SUB_BYTES + (k & 7) * 2;
                     const uint32_t buf = staging0 + (group_counter & 1u) * GROUP_BYTES;
                     const long long mg = m0 + g * 64;
-                    if (warp_has_work && POOL) {
-                        // all 64 pixels of the group for this filter, then the 16 pooled values
-                        uint32_t v[64];
+                    if (warp_has_work && POOL && p.Q == 32) {
+                        // a row pair is the whole group: the first warp of the quarter pools all 64 pixels
+                        if (half == 0) {
+                            uint32_t v[64];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + c * 16), v + c * 16);
+                            for (int c = 0; c < 4; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + c * 16), v + c * 16);
+                            tmem_ld_wait();
+                            if (k_ok) {
+                                float f[64];
+#pragma unroll
+                                for (int j = 0; j < 64; ++j) f[j] = apply_act(__uint_as_float(v[j]) + bias, p.act);
+                                uint8_t *pd = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 6) * POOL_SUB_BYTES + (k & 7) * 2;
+                                store_pooled<32, 64>(f, pd, hk, 0);
+                            }
+                        }
+                    } else if (warp_has_work && POOL) {
+                        // this warp's 32 pixels of the group (whole row pairs) for this filter, then their 8 pooled values
+                        uint32_t v[32];
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32 + c * 16), v + c * 16);
                         tmem_ld_wait();
                         if (k_ok) {
-                            float f[64];
+                            float f[32];
 #pragma unroll
-                            for (int j = 0; j < 64; ++j) f[j] = apply_act(__uint_as_float(v[j]) + bias, p.act);
+                            for (int j = 0; j < 32; ++j) f[j] = apply_act(__uint_as_float(v[j]) + bias, p.act);
                             uint8_t *pd = smem + (staging0 - base) + (group_counter & 1u) * GROUP_BYTES + (k >> 6) * POOL_SUB_BYTES + (k & 7) * 2;
                             switch (p.Q) {
-                                case 2: store_pooled<2>(f, pd, hk); break;
-                                case 4: store_pooled<4>(f, pd, hk); break;
-                                case 8: store_pooled<8>(f, pd, hk); break;
-                                case 16: store_pooled<16>(f, pd, hk); break;
-                                default: store_pooled<32>(f, pd, hk); break;
+                                case 2: store_pooled<2, 32>(f, pd, hk, half * 8); break;
+                                case 4: store_pooled<4, 32>(f, pd, hk, half * 8); break;
+                                case 8: store_pooled<8, 32>(f, pd, hk, half * 8); break;
+                                default: store_pooled<16, 32>(f, pd, hk, half * 8); break;
                             }
                         }
                     } else if (warp_has_work) {
-                        uint32_t v[64];
+                        uint32_t v[32];
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + c * 16), v + c * 16);
+                        for (int c = 0; c < 2; ++c) tmem_ld16(t_row + (uint32_t)(g * 64 + half * 32 + c * 16), v + c * 16);
                         tmem_ld_wait();
                         if (k_ok) {
 #pragma unroll
-                            for (int px = 0; px < 64; ++px) {
-                                float f = __uint_as_float(v[px]) + bias;
+                            for (int j = 0; j < 32; ++j) {
+                                float f = __uint_as_float(v[j]) + bias;
                                 f = apply_act(f, p.act);
-                                *(__nv_bfloat16 *)(dst + sub_off(px, hk)) = __float2bfloat16_rn(f);
+                                *(__nv_bfloat16 *)(dst + sub_off(half * 32 + j, hk)) = __float2bfloat16_rn(f);
                             }
                         }
                     }
