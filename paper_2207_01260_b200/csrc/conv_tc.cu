@@ -317,13 +317,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         uint32_t phase = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
-            const int tile = item / p.splits, split = item - tile * p.splits;
-            const int it_begin = split * p.ipp, it_end = min(p.iters, it_begin + p.ipp);
-            const int mt = tile / p.tiles_n, nt_f = tile - mt * p.tiles_n;
+            // the divisions below are skipped in the common cases (no split-K, one filter tile) and done in
+            // 32 bits when the pixel count allows: each costs this lone warp a few hundred cycles
+            int tile = item, split = 0, it_begin = 0, it_end = p.iters;
+            if (p.splits > 1) {
+                tile = item / p.splits; split = item - tile * p.splits;
+                it_begin = split * p.ipp; it_end = min(p.iters, it_begin + p.ipp);
+            }
+            int mt = tile, nt_f = 0;
+            if (p.tiles_n > 1) { mt = tile / p.tiles_n; nt_f = tile - mt * p.tiles_n; }
             const long long m0 = (long long)mt * p.PT;
-            const int n_img = (int)(m0 / PQ);
-            const int rem = (int)(m0 - (long long)n_img * PQ);
-            const int p0 = rem / p.Q, q0 = rem - p0 * p.Q;
+            int n_img, rem;
+            if (p.M < (1ll << 31)) {
+                n_img = (int)((uint32_t)m0 / (uint32_t)PQ);
+                rem = (int)((uint32_t)m0 - (uint32_t)n_img * (uint32_t)PQ);
+            } else {
+                n_img = (int)(m0 / PQ);
+                rem = (int)(m0 - (long long)n_img * PQ);
+            }
+            const int p0 = (int)((uint32_t)rem / (uint32_t)p.Q), q0 = rem - p0 * p.Q;
             const int wc = q0 * p.stride - p.pad, hc = p0 * p.stride - p.pad;
             if (p.small_c == 2) {
                 // stride-2 stem read as pixel pairs: the tensor map sees [N][H][W/2][16]; a pair-tap is one im2col
@@ -374,18 +386,30 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             } else {
-            for (int it = it_begin; it < it_end - (p.splits == 1 ? p.res_iters : 0); ++it) {
-                const int tap = it / p.cblks, cb = it - tap * p.cblks;
-                const int r = tap / p.S, s = tap - r * p.S;
+            // A single warp hides no latency, so this loop keeps (tap, channel block, r, s) as counters:
+            // an integer division per K block would cost more than the loads it feeds.
+            int tap = 0, cb = 0, r = 0, s = 0;
+            if (it_begin) {
+                tap = it_begin / p.cblks; cb = it_begin - tap * p.cblks;
+                r = tap / p.S; s = tap - r * p.S;
+            }
+            const int it_last = it_end - (p.splits == 1 ? p.res_iters : 0);
+            const int k0 = nt_f * p.FT;
+            for (int it = it_begin; it < it_last; ++it) {
                 ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                 if (!ok) break;
                 if (elect_one()) {
                     const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
-                    mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
-                    tma_load_im2col(x_dst, &tm_x, full_bar(stage), cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
-                    tma_load_3d(x_dst + x_bytes, &tm_w, full_bar(stage), cb * BK, tap, nt_f * p.FT);
+                    const uint32_t fb = full_bar(stage);
+                    mbar_expect_tx(fb, (uint32_t)stage_bytes);
+                    tma_load_im2col(x_dst, &tm_x, fb, cb * BK, wc, hc, n_img, (uint16_t)s, (uint16_t)r);
+                    tma_load_3d(x_dst + x_bytes, &tm_w, fb, cb * BK, tap, k0);
                 }
                 __syncwarp();
+                if (++cb == p.cblks) {
+                    cb = 0; ++tap;
+                    if (++s == p.S) { s = 0; ++r; }
+                }
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
             }
@@ -413,9 +437,22 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         int stage = 0, acc = 0;
         uint32_t phase = 0, acc_phase = 0;
         bool ok = true;
+        // This warp, too, runs alone on its scheduler: the loop below keeps the channel-block counter and the
+        // operand descriptors of the current stage incrementally (no division, no descriptor rebuild per K block).
+        const uint64_t dx0 = smem_desc_sw128(base), dw0 = smem_desc_sw128(base + (uint32_t)x_bytes);
+        const uint64_t stage_step = (uint64_t)(stage_bytes >> 4);     // descriptor start addresses count 16-byte units
+        uint64_t dx = dx0, dw = dw0;
+        const int main_iters = p.iters - p.res_iters;
+        const bool plain = p.small_c == 0;
         for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
-            const int split = item % p.splits;
-            const int it_begin = split * p.ipp, it_end = min(p.iters, it_begin + p.ipp);
+            int it_begin = 0, it_end = p.iters;
+            int cb = 0;
+            if (p.splits > 1) {
+                const int split = item % p.splits;
+                it_begin = split * p.ipp;
+                it_end = min(p.iters, it_begin + p.ipp);
+                cb = it_begin % p.cblks;
+            }
             ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
@@ -424,63 +461,72 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             for (int it = it_begin; it < it_end; ++it) {
                 ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag, p.status));
                 if (!ok) break;
-                const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
-                const uint64_t dw = smem_desc_sw128(x_addr + x_bytes);
-                int nk;
-                const int main_iters = p.iters - p.res_iters;
                 const bool res_it = it >= main_iters;
-                if (res_it) {
-                    int left = p.k_pad - (it - main_iters) * BK;
-                    if (left > BK) left = BK;
-                    nk = (left + 15) >> 4;
-                } else if (p.small_c == 2) {
-                    nk = p.R * p.pair_taps - it * 4;
-                    if (nk > 4) nk = 4;
-                } else if (p.small_c) {
-                    int nt = p.R * p.S - it * 8;
-                    if (nt > 8) nt = 8;
-                    nk = (nt + 1) >> 1;
-                } else {
-                    nk = ((it + 1) % p.cblks == 0) ? p.ksteps_last : BK / 16;
-                }
-                if (elect_one()) {
-                    if (p.small_c == 2 && !res_it) {
-                        // pixel operand: one pair-tap (16 channels) per MMA, pair-taps PT*32 bytes apart
-                        for (int kk = 0; kk < nk; ++kk) {
-                            const uint64_t dxp = smem_desc_sw32(x_addr + (uint32_t)kk * (uint32_t)p.PT * 32u);
-                            if (ORIENT == ORIENT_PIX)
-                                umma_bf16(d_tmem, dxp, dw + (uint64_t)(2 * kk), idesc, accumulate);
-                            else
-                                umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dxp, idesc, accumulate);
-                            accumulate = 1;
-                        }
-                    } else if (p.small_c && !res_it) {
-                        // pixel operand: two taps (2 x 8 channels) per MMA, taps PT*16 bytes apart
-                        const uint32_t tap_bytes = (uint32_t)p.PT * 16u;
-                        for (int kk = 0; kk < nk; ++kk) {
-                            const uint64_t dxi = smem_desc_interleaved(x_addr + (uint32_t)(2 * kk) * tap_bytes, tap_bytes);
-                            if (ORIENT == ORIENT_PIX)
-                                umma_bf16(d_tmem, dxi, dw + (uint64_t)(2 * kk), idesc, accumulate);
-                            else
-                                umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dxi, idesc, accumulate);
-                            accumulate = 1;
-                        }
-                    } else {
-                        const uint64_t dx = smem_desc_sw128(x_addr);
-                        for (int kk = 0; kk < nk; ++kk) {
-                            // 16 channels = 32 bytes further along the swizzled row: +2 in 16-byte units
-                            if (ORIENT == ORIENT_PIX)
-                                umma_bf16(d_tmem, dx + (uint64_t)(2 * kk), dw + (uint64_t)(2 * kk), idesc, accumulate);
-                            else
-                                umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dx + (uint64_t)(2 * kk), idesc, accumulate);
-                            accumulate = 1;
-                        }
+                if (plain || res_it) {
+                    int nk = BK / 16;
+                    if (res_it) {
+                        int left = p.k_pad - (it - main_iters) * BK;
+                        if (left > BK) left = BK;
+                        nk = (left + 15) >> 4;
+                    } else if (cb == p.cblks - 1) {
+                        nk = p.ksteps_last;
                     }
-                    umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    if (elect_one()) {
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk) {
+                            if (kk < nk) {
+                                // 16 channels = 32 bytes further along the swizzled row: +2 in 16-byte units
+                                if (ORIENT == ORIENT_PIX)
+                                    umma_bf16(d_tmem, dx + (uint64_t)(2 * kk), dw + (uint64_t)(2 * kk), idesc, accumulate);
+                                else
+                                    umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dx + (uint64_t)(2 * kk), idesc, accumulate);
+                                accumulate = 1;
+                            }
+                        }
+                        umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    }
+                } else {
+                    const uint32_t x_addr = base + (uint32_t)stage * stage_bytes;
+                    int nk;
+                    if (p.small_c == 2) {
+                        nk = p.R * p.pair_taps - it * 4;
+                        if (nk > 4) nk = 4;
+                    } else {
+                        int nt = p.R * p.S - it * 8;
+                        if (nt > 8) nt = 8;
+                        nk = (nt + 1) >> 1;
+                    }
+                    if (elect_one()) {
+                        if (p.small_c == 2) {
+                            // pixel operand: one pair-tap (16 channels) per MMA, pair-taps PT*32 bytes apart
+                            for (int kk = 0; kk < nk; ++kk) {
+                                const uint64_t dxp = smem_desc_sw32(x_addr + (uint32_t)kk * (uint32_t)p.PT * 32u);
+                                if (ORIENT == ORIENT_PIX)
+                                    umma_bf16(d_tmem, dxp, dw + (uint64_t)(2 * kk), idesc, accumulate);
+                                else
+                                    umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dxp, idesc, accumulate);
+                                accumulate = 1;
+                            }
+                        } else {
+                            // pixel operand: two taps (2 x 8 channels) per MMA, taps PT*16 bytes apart
+                            const uint32_t tap_bytes = (uint32_t)p.PT * 16u;
+                            for (int kk = 0; kk < nk; ++kk) {
+                                const uint64_t dxi = smem_desc_interleaved(x_addr + (uint32_t)(2 * kk) * tap_bytes, tap_bytes);
+                                if (ORIENT == ORIENT_PIX)
+                                    umma_bf16(d_tmem, dxi, dw + (uint64_t)(2 * kk), idesc, accumulate);
+                                else
+                                    umma_bf16(d_tmem, dw + (uint64_t)(2 * kk), dxi, idesc, accumulate);
+                                accumulate = 1;
+                            }
+                        }
+                        umma_commit(empty_bar(stage));
+                    }
                 }
                 accumulate = 1;
                 __syncwarp();
-                if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                if (++cb == p.cblks) cb = 0;
+                dx += stage_step; dw += stage_step;
+                if (++stage == p.stages) { stage = 0; phase ^= 1u; dx = dx0; dw = dw0; }
             }
             if (ok && elect_one()) umma_commit(tfull_bar(acc));
             __syncwarp();
@@ -512,8 +558,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             return r;
         };
         for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
-            const int tile = item / p.splits, split = item - tile * p.splits;
-            const int mt = tile / p.tiles_n, nt = tile - mt * p.tiles_n;
+            int tile = item, split = 0;
+            if (p.splits > 1) { tile = item / p.splits; split = item - tile * p.splits; }
+            int mt = tile, nt = 0;
+            if (p.tiles_n > 1) { mt = tile / p.tiles_n; nt = tile - mt * p.tiles_n; }
             const long long m0 = (long long)mt * p.PT;
             const int k_base = nt * p.FT;
             // the epilogue ignores the abort flag: all eight warps must take the same decisions,
