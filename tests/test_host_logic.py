@@ -54,6 +54,10 @@ def test_plan_shapes_and_families(cp):
     assert cp.KERNEL_NAMES[p.kernel] == "depthwise" and (p.P, p.Q) == (28, 28) and p.c_pad == 112
     assert p.flops == 2.0 * 8 * 108 * 28 * 28 * 9
     p = cp.cprune_task_plan(128, 45, 32, 32, 58, 3, 3, 1, 1, pool="max2x2")
+    # the pool runs inside the conv kernel: the output is the pooled tensor and no unpooled copy is kept
+    assert (p.out_h, p.out_w) == (16, 16) and p.workspace_bytes == 0
+    # the CUDA-core family does not fuse it: the unpooled output goes to the workspace
+    p = cp.cprune_task_plan(128, 45, 32, 32, 58, 3, 3, 1, 1, pool="max2x2", kernel="direct")
     assert (p.out_h, p.out_w) == (16, 16) and p.workspace_bytes == 128 * 32 * 32 * 64 * 2
     # every pruned filter count gets a legal tile: N tile a multiple of 16 within the accumulator
     for K in range(64, 513, 7):
