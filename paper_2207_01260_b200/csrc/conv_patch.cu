@@ -1,0 +1,606 @@
+// Stride-1 dense conv task (3x3 and other R x S > 1) on the sm_100a tensor cores with the input
+// patch kept in shared memory (paper Sec. 3.4: a task is Conv2d + folded BatchNorm + activation;
+// Sec. 3.5: the filter count is whatever pruning left).
+//
+// Why a second tensor-core kernel: the im2col kernel (conv_tc.cu) writes every activation element
+// R*S times into shared memory, and on this GPU the shared-memory port (128 bytes per clock: TMA
+// writes plus the operand reads of tcgen05.mma) is what bounds it, not the tensor pipe.  Here a
+// tile is TH whole output rows of one image.  Its input patch, (TH + R - 1) x (W + 2 pad) pixels x
+// 64 channels, is loaded ONCE per channel block by one tiled TMA load (out-of-range pixels and
+// channels arrive as zeros, which is the padding).  The patch sits in shared memory as rows of
+// 128 bytes, one per pixel, in row-major order of the padded image, 128-byte swizzled.  For filter
+// tap (r, s) the pixel operand of the MMA is the same patch read from a start address
+// (r * Wp + s) * 128 bytes further on (Wp = W + 2 pad): the swizzle is a function of the
+// shared-memory address, so a descriptor may start at any 128-byte row (checked on B200).
+//
+// The accumulator row of a pixel is its "slot" i * Wp + j (i row in the tile, j column); slots with
+// j >= Q are the S - 1 wrap-around columns: they are computed and thrown away.  A tile has MT
+// blocks of 128 slots (MT = 1 or 2, one accumulator each, both fed by the same filter stage).
+//
+//   warp 0       patch loads (one per channel block);
+//   warps 1, 2   filter loads, one per (channel block, tap), taken in turn; small filter sets
+//                stay resident in shared memory for the whole kernel;
+//   warps 3, 12  tcgen05.mma issue, one warp per accumulator block;
+//   warps 4..11  epilogue: tcgen05.ld, bias (+ residual), activation, bf16 into a swizzled staging
+//                buffer, then all 256 threads copy the valid pixels out with 16-byte stores, eight
+//                threads per pixel (whole 128-byte lines; stores of 16 bytes per thread at a pixel
+//                stride were measured to be several times slower); a 2x2 max-pool is taken while
+//                copying.
+// Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA raises STATUS_TIMEOUT and leaves.
+#include <cuda.h>
+
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "plan.h"
+#include "sm100_ptx.cuh"
+
+namespace cprune {
+
+constexpr int PK_THREADS = 13 * 32;
+constexpr int PK_MMA_WARP = 3;
+constexpr int PK_FIRST_EPI = 4;
+constexpr int PK_MMA_WARP2 = 12;         // issues for the second accumulator block when MT = 2
+constexpr int PK_MAX_WSTAGES = 32;
+constexpr int PK_PATCH_STAGES = 2;
+constexpr int PK_CTRL_BYTES = 3072;      // barriers (1 KB) + slot table (2 KB)
+constexpr int PK_BLOCK_BYTES = 16384;    // staged block: 128 slots x 64 filters bf16
+
+struct PatchParams {
+    int P, Q, Wp, TH, tiles_per_img, tiles_m, tiles_n;
+    int FT, MT, R, S, pad, cblks, ksteps_last, k_pad;
+    int act, wstages, resident, acc_bufs, staging_bufs, pool;
+    int patch_bytes;       // shared memory of one patch stage
+    int patch_box_bytes;   // bytes one patch load delivers
+    const float *bias;
+    const __nv_bfloat16 *res;
+    __nv_bfloat16 *y;
+    int *status;
+};
+
+__device__ __forceinline__ uint4 bf16x8_max(uint4 a, uint4 b) {
+    uint4 r;
+    __nv_bfloat162 *pa = reinterpret_cast<__nv_bfloat162 *>(&a), *pb = reinterpret_cast<__nv_bfloat162 *>(&b);
+    __nv_bfloat162 *pr = reinterpret_cast<__nv_bfloat162 *>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pr[i] = __hmax2(pa[i], pb[i]);
+    return r;
+}
+
+// All MMAs of one filter tap: for each of the MT accumulator blocks, nk steps of 16 channels.  a_lo and w_lo are
+// the low words of the operand descriptors (start address in 16-byte units).  Called by the whole warp: the
+// operands are computed by all lanes (they stay in uniform registers) and one elected lane issues.
+template <int MT>
+__device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint32_t FT, uint32_t a_lo, uint32_t w_lo, uint32_t idesc,
+                                          uint32_t accumulate, int nk, uint32_t commit_w, uint32_t commit_p) {
+    uint32_t al[MT][4], wl[4], dd[MT];
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) wl[kk] = w_lo + (uint32_t)(2 * kk);
+#pragma unroll
+    for (int mb = 0; mb < MT; ++mb) {
+        dd[mb] = d_tmem + (uint32_t)mb * FT;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) al[mb][kk] = a_lo + (uint32_t)(mb * 1024 + 2 * kk);
+    }
+    if (elect_one()) {
+        if (nk == 4) {
+#pragma unroll
+            for (int mb = 0; mb < MT; ++mb)
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16_sw128(dd[mb], al[mb][kk], wl[kk], idesc, kk ? 1u : accumulate);
+        } else {
+#pragma unroll
+            for (int mb = 0; mb < MT; ++mb)
+#pragma unroll
+                for (int kk = 0; kk < 3; ++kk)
+                    if (kk < nk) umma_bf16_sw128(dd[mb], al[mb][kk], wl[kk], idesc, kk ? 1u : accumulate);
+        }
+        if (commit_w) umma_commit(commit_w);
+        if (commit_p) umma_commit(commit_p);
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(PK_THREADS, 1)
+conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                  const __grid_constant__ CUtensorMap tm_y, const PatchParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t w_bytes = (uint32_t)p.FT * 128u;
+    const uint32_t patch0 = base;
+    const uint32_t w0 = patch0 + PK_PATCH_STAGES * (uint32_t)p.patch_bytes;
+    const uint32_t staging0 = w0 + (uint32_t)p.wstages * w_bytes;
+    const uint32_t stage_buf_bytes = (uint32_t)p.MT * PK_BLOCK_BYTES;
+    const uint32_t ctrl0 = staging0 + (uint32_t)p.staging_bufs * stage_buf_bytes;
+    uint8_t *ctrl = smem + (ctrl0 - base);
+    auto pfull = [&](int s) { return ctrl0 + 8u * s; };
+    auto pempty = [&](int s) { return ctrl0 + 16u + 8u * s; };
+    auto tfull = [&](int a) { return ctrl0 + 32u + 8u * a; };
+    auto tempty = [&](int a) { return ctrl0 + 48u + 8u * a; };
+    const uint32_t epi_bar = ctrl0 + 64u;
+    uint32_t *tmem_slot = (uint32_t *)(ctrl + 72);
+    volatile int *abort_flag = (volatile int *)(ctrl + 76);
+    auto wfull = [&](int s) { return ctrl0 + 128u + 8u * s; };
+    auto wempty = [&](int s) { return ctrl0 + 384u + 8u * s; };
+    int2 *lut = (int2 *)(ctrl + 1024);   // entry -> (source slot | tile row << 16, output offset in elements); x < 0: nothing to store
+
+    // the shuffle tells the compiler that the warp number is the same in all lanes, so that the role code below
+    // (loop counters, descriptors, TMA coordinates) can live in uniform registers
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+    const int RS = p.R * p.S;
+
+    if (threadIdx.x == 0) {
+        // every accumulator block has its own issuing warp: stages are free, and a tile is complete, once all have committed
+        for (int s = 0; s < PK_PATCH_STAGES; ++s) { mbar_init(pfull(s), 1); mbar_init(pempty(s), p.MT); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull(a), p.MT); mbar_init(tempty(a), 8); }
+        for (int s = 0; s < p.wstages; ++s) { mbar_init(wfull(s), 1); mbar_init(wempty(s), p.MT); }
+        mbar_init(epi_bar, 8);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // slot table: which accumulator rows hold real output pixels and where they go
+    for (int e = threadIdx.x; e < 256; e += PK_THREADS) {
+        int2 v = make_int2(-1, 0);
+        if (!p.pool) {
+            const int i = e / p.Wp, j = e - i * p.Wp;
+            if (e < 128 * p.MT && j < p.Q && i < p.TH) v = make_int2(e | (i << 16), (i * p.Q + j) * p.k_pad);
+        } else {
+            const int hq = p.Q >> 1;
+            const int i2 = e / hq, j2 = e - i2 * hq;
+            if (i2 < (p.TH >> 1)) v = make_int2((2 * i2 * p.Wp + 2 * j2) | ((2 * i2) << 16), (i2 * hq + j2) * p.k_pad);
+        }
+        lut[e] = v;
+    }
+    if (warp == PK_MMA_WARP) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int total_items = p.tiles_m * p.tiles_n;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ patch loads
+        int ps = 0;
+        uint32_t pphase = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            int tm = item;
+            if (p.tiles_n > 1) tm = item / p.tiles_n;
+            const int n = tm / p.tiles_per_img;
+            const int p0 = (tm - n * p.tiles_per_img) * p.TH;
+            for (int cb = 0; cb < p.cblks; ++cb) {
+                ok = __all_sync(0xffffffffu, mbar_wait(pempty(ps), pphase ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                if (elect_one()) {
+                    mbar_expect_tx(pfull(ps), (uint32_t)p.patch_box_bytes);
+                    tma_load_4d(patch0 + (uint32_t)ps * p.patch_bytes, &tm_x, pfull(ps), cb * 64, -p.pad, p0 - p.pad, n);
+                }
+                __syncwarp();
+                if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; }
+            }
+        }
+    } else if (warp < PK_MMA_WARP) {
+        // ------------------------------------------------------------------ filter loads
+        int ws = 0, turn = 0;
+        uint32_t wphase = 0;
+        bool ok = true;
+        const int me = warp - 1;
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            if (p.resident && item != (int)blockIdx.x) break;     // the filters of the first tile stay
+            int nt = 0;
+            if (p.tiles_n > 1) nt = item % p.tiles_n;
+            const int k0 = nt * p.FT;
+            for (int cb = 0; cb < p.cblks && ok; ++cb) {
+                for (int tap = 0; tap < RS; ++tap) {
+                    const bool mine = turn == me;
+                    turn ^= 1;
+                    if (mine) {
+                        if (!p.resident) ok = __all_sync(0xffffffffu, mbar_wait(wempty(ws), wphase ^ 1u, abort_flag, p.status));
+                        if (!ok) break;
+                        if (elect_one()) {
+                            mbar_expect_tx(wfull(ws), w_bytes);
+                            tma_load_3d(w0 + (uint32_t)ws * w_bytes, &tm_w, wfull(ws), cb * 64, tap, k0);
+                        }
+                        __syncwarp();
+                    }
+                    if (++ws == p.wstages) { ws = 0; wphase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == PK_MMA_WARP || warp == PK_MMA_WARP2) {
+        // ------------------------------------------------------------------ MMA issue
+        // tcgen05.mma issue is close to synchronous (about two instructions may be pending, measured), so the
+        // bookkeeping between taps would leave the tensor pipe idle if one warp issued everything: with MT = 2
+        // each accumulator block gets its own issuing warp and the two interleave.
+        const int mb = warp == PK_MMA_WARP ? 0 : 1;
+        if (mb < p.MT) {
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.FT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        int ps = 0, ws = 0, acc = 0;
+        uint32_t pphase = 0, wphase = 0, acc_phase = 0;
+        bool ok = true;
+        // A lone warp pays several cycles for every instruction, so the loop works on the low descriptor words
+        // only (32-bit adds) and issues a tap's MMAs from fully unrolled code.
+        const uint32_t patch_lo0 = desc_lo_sw128(patch0), w_lo0 = desc_lo_sw128(w0);
+        const uint32_t patch_step = (uint32_t)p.patch_bytes >> 4, w_step = w_bytes >> 4;
+        const uint32_t row_step = (uint32_t)((p.Wp - p.S + 1) * 8);   // descriptor units (16 bytes) from tap (r, S-1) to (r+1, 0)
+        uint32_t patch_lo = patch_lo0, w_lo = w_lo0;
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            ok = __all_sync(0xffffffffu, mbar_wait(tempty(acc), acc_phase ^ 1u, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)((acc * p.MT + mb) * p.FT);
+            uint32_t accumulate = 0;
+            for (int cb = 0; cb < p.cblks && ok; ++cb) {
+                ok = __all_sync(0xffffffffu, mbar_wait(pfull(ps), pphase, abort_flag, p.status));
+                if (!ok) break;
+                const int nk = cb == p.cblks - 1 ? p.ksteps_last : 4;
+                uint32_t tap_lo = patch_lo + (uint32_t)(mb * 1024);      // the second block's slots start 16 KB further on
+                int s = 0;
+                for (int tap = 0; tap < RS; ++tap) {
+                    // resident filters: the barrier completes once (first tile) and stays complete for parity 0
+                    ok = __all_sync(0xffffffffu, mbar_wait(wfull(ws), p.resident ? 0u : wphase, abort_flag, p.status));
+                    if (!ok) break;
+                    {
+                        const uint32_t cw = p.resident ? 0u : wempty(ws), cp = tap == RS - 1 ? pempty(ps) : 0u;
+                        issue_tap<1>(d_tmem, (uint32_t)p.FT, tap_lo, w_lo, idesc, accumulate, nk, cw, cp);
+                    }
+                    accumulate = 1;
+                    w_lo += w_step;
+                    if (++ws == p.wstages) { ws = 0; wphase ^= 1u; w_lo = w_lo0; }
+                    tap_lo += 8;
+                    if (++s == p.S) { s = 0; tap_lo += row_step - 8; }
+                }
+                patch_lo += patch_step;
+                if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; patch_lo = patch_lo0; }
+            }
+            if (ok && elect_one()) umma_commit(tfull(acc));
+            __syncwarp();
+            if (p.acc_bufs == 2) { if (++acc == 2) { acc = 0; acc_phase ^= 1u; } }
+            else acc_phase ^= 1u;
+        }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;
+        const int half = (warp - PK_FIRST_EPI) >> 2;
+        const int trow = quarter * 32 + lane;          // accumulator lane = slot within its 128-slot block
+        const int etid = threadIdx.x - PK_FIRST_EPI * 32;
+        int acc = 0;
+        uint32_t acc_phase = 0, epi_phase = 0, group_counter = 0;
+        bool ok = true;
+        auto epi_sync = [&]() {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(epi_bar);
+            bool r = __all_sync(0xffffffffu, mbar_wait(epi_bar, epi_phase, abort_flag, p.status, false));
+            epi_phase ^= 1u;
+            return r;
+        };
+        // this thread's slot in each accumulator block never changes: where its pixel goes (elements from the tile's
+        // first pixel) and which tile row it is in; x < 0: a wrap-around or unused slot
+        const int2 my_slot[2] = {lut[trow], lut[128 + trow]};
+        // activation as a clamp: no branches in the per-element code
+        const float act_lo = p.act == CPRUNE_ACT_NONE ? -INFINITY : 0.f, act_hi = p.act == CPRUNE_ACT_RELU6 ? 6.f : INFINITY;
+        const bool store_thread = warp == PK_FIRST_EPI && lane == 0;
+        const int groups = (p.FT + 63) / 64;
+        const int n_entries = p.pool ? (p.TH >> 1) * (p.Q >> 1) : 128 * p.MT;
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            int tm = item, nt = 0;
+            if (p.tiles_n > 1) { tm = item / p.tiles_n; nt = item - tm * p.tiles_n; }
+            const int n = tm / p.tiles_per_img;
+            const int p0 = (tm - n * p.tiles_per_img) * p.TH;
+            const int k0 = nt * p.FT;
+            const int rows_valid = p.P - p0;                 // tile rows below this are real image rows
+            const size_t in_tile = ((size_t)n * p.P + p0) * p.Q * p.k_pad;
+            __nv_bfloat16 *ytile = p.pool ? p.y + ((size_t)n * (p.P >> 1) + (p0 >> 1)) * (p.Q >> 1) * p.k_pad : p.y + in_tile;
+            ok = __all_sync(0xffffffffu, mbar_wait(tfull(acc), acc_phase, abort_flag, p.status, false));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.MT * p.FT);
+            for (int g = 0; g < groups && ok; ++g) {
+                const uint32_t boff = (p.staging_bufs == 2 ? (group_counter & 1u) : 0u) * stage_buf_bytes;
+                uint8_t *buf = smem + (staging0 - base) + boff;
+                const int ch = g * 64 + half * 32;           // this warp's 32 filters of the group
+                for (int mb = 0; mb < p.MT; ++mb) {
+                    const int slot = mb * 128 + trow;
+                    uint32_t v[32];
+#pragma unroll
+                    for (int sb = 0; sb < 2; ++sb)
+                        if (ch + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(mb * p.FT + ch + sb * 16), v + sb * 16);
+                    bf16x8 rv[4];
+                    const int2 ms = my_slot[mb];
+                    const bool px_ok = !p.pool && ms.x >= 0 && (ms.x >> 16) < rows_valid;
+                    const bool has_res = p.res != nullptr && px_ok;
+                    if (has_res) {
+                        const __nv_bfloat16 *rrow = p.res + in_tile + ms.y + k0 + ch;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (k0 + ch + j * 8 < p.k_pad) rv[j] = ldg8((const bf16x8 *)(rrow + j * 8));
+                    }
+                    tmem_ld_wait();
+                    if (g == groups - 1 && mb == p.MT - 1) {     // accumulator fully read: hand it back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty(acc));
+                    }
+#pragma unroll
+                    for (int sb = 0; sb < 2; ++sb) {
+                        const int c0 = ch + sb * 16;
+                        if (c0 < p.FT) {
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float f[8];
+                                const float4 b0 = __ldg((const float4 *)(p.bias + k0 + c0 + h * 8));
+                                const float4 b1 = __ldg((const float4 *)(p.bias + k0 + c0 + h * 8 + 4));
+                                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[sb * 16 + h * 8 + j]) + bb[j];
+                                if (has_res && k0 + c0 + h * 8 < p.k_pad) {
+                                    float rf[8];
+                                    unpack8(rv[sb * 2 + h], rf);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) f[j] += rf[j];
+                                }
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) f[j] = fminf(fmaxf(f[j], act_lo), act_hi);
+                                *(bf16x8 *)(buf + mb * PK_BLOCK_BYTES + sub_off(trow, half * 4 + sb * 2 + h)) = pack8(f);
+                            }
+                        }
+                    }
+                }
+                if (!p.pool) {
+                    // one TMA store per group: the staged slots are TH rows of Wp pixels; the tensor map's box has
+                    // that shape, and the wrap-around columns (j >= Q), rows below the image and filters beyond
+                    // k_pad fall outside the tensor, where a store writes nothing
+                    fence_async_smem();
+                    // the buffer written next (the other one) was last read by the previous group's store
+                    if (p.staging_bufs == 2 && store_thread) tma_store_wait_read<0>();
+                    ok = epi_sync();
+                    if (!ok) break;
+                    if (store_thread) {
+                        if (k0 + g * 64 < p.k_pad) tma_store_4d(&tm_y, staging0 + boff, k0 + g * 64, 0, p0, n);
+                        tma_store_commit();
+                        if (p.staging_bufs == 1) tma_store_wait_read<0>();
+                    }
+                    if (p.staging_bufs == 1) {
+                        ok = epi_sync();
+                        if (!ok) break;
+                    }
+                    ++group_counter;
+                    continue;
+                }
+                ok = epi_sync();
+                if (!ok) break;
+                // copy-out: eight threads per output pixel, 16 bytes each
+                const int kg = k0 + g * 64;
+                for (int e = etid; e < n_entries * 8; e += 256) {
+                    const int2 l = lut[e >> 3];
+                    const int chunk = e & 7;
+                    if (l.x >= 0 && (l.x >> 16) < rows_valid && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
+                        const int slot = l.x & 0xffff;
+                        auto staged = [&](int sl) { return *(const uint4 *)(buf + (sl >> 7) * PK_BLOCK_BYTES + sub_off(sl & 127, chunk)); };
+                        uint4 val = bf16x8_max(staged(slot), staged(slot + 1));
+                        val = bf16x8_max(val, bf16x8_max(staged(slot + p.Wp), staged(slot + p.Wp + 1)));
+                        *(uint4 *)(ytile + l.y + kg + chunk * 8) = val;
+                    }
+                }
+                if (p.staging_bufs == 1) {
+                    ok = epi_sync();
+                    if (!ok) break;
+                }
+                ++group_counter;
+            }
+            if (p.acc_bufs == 2) { if (++acc == 2) { acc = 0; acc_phase ^= 1u; } }
+            else acc_phase ^= 1u;
+        }
+        if (store_thread) tma_store_wait_all();      // staged data must be read before the CTA's memory goes away
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);   // let copies in flight land before the memory goes away
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == PK_MMA_WARP) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host
+
+// Estimated cycles of one tile.  Per tcgen05.mma (M = 128, N = FT, K = 16) the tensor pipe needs FT / 2 cycles
+// and the operand reads (128 + FT) * 32 bytes of the 128 bytes per clock that shared memory delivers; the TMA
+// writes of filters and patches share that port (measured on B200).
+static double tile_cycles(int MT, int FT, int RS, int cblks, int ksteps_last, int Wp, int TH, int R, bool resident,
+                          int acc_bufs) {
+    double total = 0;
+    for (int cb = 0; cb < cblks; ++cb) {
+        const int nk = cb == cblks - 1 ? ksteps_last : 4;
+        const double tensor = MT * nk * (FT / 2.0);
+        const double smem = (MT * nk * (128.0 + FT) * 32.0 + (resident ? 0.0 : FT * 128.0)) / 128.0;
+        total += RS * (tensor > smem ? tensor : smem) + Wp * (TH + R - 1);
+    }
+    const double epilogue = MT * ((FT + 63) / 64) * 500.0;
+    return total + (acc_bufs == 2 ? (epilogue > total ? epilogue - total : 0.0) : epilogue) + 1500.0;
+}
+
+// Decides whether the task runs on the patch kernel and with which tiling; fills plan->info tile fields.
+cprune_status plan_conv_patch(cprune_plan *plan) {
+    cprune_plan_info &i = plan->info;
+    plan->patch = 0;
+    if (i.groups != 1 || i.stride != 1 || i.R * i.S <= 1 || i.R > 7 || i.S > 7) return CPRUNE_ERR_UNSUPPORTED;
+    if (i.c_pad < 16) return CPRUNE_ERR_UNSUPPORTED;
+    const int Wp = i.W + 2 * i.pad;
+    if (Wp > 128 || i.Q != Wp - i.S + 1 || i.H + 2 * i.pad - i.R + 1 != i.P) return CPRUNE_ERR_UNSUPPORTED;
+    const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
+    if (pool && (plan->opts.residual || (i.P & 1) || (i.Q & 1))) return CPRUNE_ERR_UNSUPPORTED;
+    const int k16 = round_up(i.K, 16);
+    const int cblks = (i.c_pad + 63) / 64;
+    const int ksteps_last = (i.c_pad - (cblks - 1) * 64 + 15) / 16;
+    const int RS = i.R * i.S;
+    double best = 1e30;
+    PatchTiling bt = {};
+    const char *force_mt = getenv("CPRUNE_PATCH_MT");       // measurement overrides
+    const char *force_tn = getenv("CPRUNE_PATCH_TN");
+    for (int MT = 1; MT <= 2; ++MT) {
+        if (force_mt && atoi(force_mt) != MT) continue;
+        int TH = (128 * MT) / Wp;
+        if (TH > i.P) TH = i.P;
+        if (pool) TH &= ~1;
+        if (TH < 1) continue;
+        const int tiles_per_img = (i.P + TH - 1) / TH;
+        for (int tiles_n = 1; tiles_n <= 8; ++tiles_n) {
+            if (force_tn && atoi(force_tn) != tiles_n) continue;
+            // with several filter tiles every tile ends on a 64-filter boundary: the stores are 64 filters wide and
+            // only the tensor's own edge clips them
+            const int FT = round_up((k16 + tiles_n - 1) / tiles_n, tiles_n > 1 ? 64 : 16);
+            if (FT > 256 || MT * FT > 512) continue;
+            if ((k16 + FT - 1) / FT != tiles_n) continue;
+            const int acc_bufs = 2 * MT * FT <= 512 ? 2 : 1;
+            const int patch_bytes = round_up((128 * MT + (i.R - 1) * Wp + i.S - 1) * 128, 1024);
+            if (patch_bytes < Wp * (TH + i.R - 1) * 128) continue;
+            const int fixed = 1024 + PK_PATCH_STAGES * patch_bytes + PK_CTRL_BYTES;
+            const int budget = 227 * 1024 - fixed;
+            const int sb_max = 2, sb_min = 1;
+            int staging_bufs = sb_max, wstages = 0, resident = 0;
+            // resident filters when the whole set of this filter tile fits
+            if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES) {
+                for (int sb = sb_max; sb >= sb_min && !resident; --sb)
+                    if (RS * cblks * FT * 128 + sb * MT * PK_BLOCK_BYTES <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
+            }
+            if (!resident) {
+                staging_bufs = sb_max;
+                wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / (FT * 128);
+                if (wstages < 3 && sb_min < sb_max) {
+                    staging_bufs = sb_min;
+                    wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / (FT * 128);
+                }
+                if (wstages < 3) continue;
+                if (wstages > 8) wstages = 8;
+            }
+            const long long tiles = (long long)i.N * tiles_per_img * tiles_n;
+            const double waves = (double)((tiles + 147) / 148);
+            double t = waves * tile_cycles(MT, FT, RS, cblks, ksteps_last, Wp, TH, i.R, resident != 0, acc_bufs);
+            if (resident) t += RS * cblks * FT;    // one-time filter load
+            if (t < best) {
+                best = t;
+                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes};
+            }
+        }
+    }
+    if (best >= 1e30) return CPRUNE_ERR_UNSUPPORTED;
+    // share of accumulator rows that hold real pixels; below one half the im2col kernel is the better choice
+    const double fill = (double)i.P * i.Q / ((double)bt.tiles_per_img * 128 * bt.MT);
+    if (fill < 0.5) return CPRUNE_ERR_UNSUPPORTED;
+    // too few tiles for the SMs: the im2col kernel can split the reduction over more CTAs
+    if ((long long)i.N * bt.tiles_per_img * bt.tiles_n < 64) return CPRUNE_ERR_UNSUPPORTED;
+    plan->patch = 1;
+    plan->pt = bt;
+    plan->orient = 0;
+    plan->small_c = 0;
+    plan->s_packed = i.S;
+    plan->splits = 1;
+    plan->ipp = 0;
+    plan->partial_bytes = 0;
+    plan->fused_pool = pool ? 1 : 0;
+    i.tile_m = 128 * bt.MT;
+    i.tile_n = bt.FT;
+    i.tile_k = 64;
+    i.stages = bt.wstages;
+    i.tiles_m = i.N * bt.tiles_per_img;
+    i.tiles_n = bt.tiles_n;
+    i.k_alloc = bt.tiles_n * bt.FT;
+    const int ksteps = (cblks - 1) * 4 + ksteps_last;
+    i.padded_flops = 2.0 * (double)i.tiles_m * i.tile_m * (double)i.k_alloc * RS * ksteps * 16.0;
+    plan->smem_bytes = 1024 + PK_PATCH_STAGES * bt.patch_bytes + bt.wstages * bt.FT * 128 + bt.staging_bufs * bt.MT * PK_BLOCK_BYTES +
+                       PK_CTRL_BYTES;
+    return CPRUNE_OK;
+}
+
+cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res, void *y,
+                                cudaStream_t st) {
+    const cprune_plan_info &i = plan->info;
+    const PatchTiling &t = plan->pt;
+    const int Wp = i.W + 2 * i.pad;
+    CUtensorMap tm_x, tm_w, tm_y;
+    {
+        std::lock_guard<std::mutex> lock(plan->mu);
+        if (plan->map_x != x) {
+            const unsigned long long dims[4] = {(unsigned long long)i.c_pad, (unsigned long long)i.W, (unsigned long long)i.H,
+                                                (unsigned long long)i.N};
+            const unsigned long long strides[3] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.W * i.c_pad * 2,
+                                                   (unsigned long long)i.H * i.W * i.c_pad * 2};
+            const unsigned box[4] = {64, (unsigned)Wp, (unsigned)(t.TH + i.R - 1), 1};
+            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_a, x, 4, dims, strides, box);
+            if (s != CPRUNE_OK) return s;
+            plan->map_x = x;
+        }
+        if (plan->map_w != w) {
+            const unsigned long long dims[3] = {(unsigned long long)i.c_pad, (unsigned long long)(i.R * i.S), (unsigned long long)i.k_alloc};
+            const unsigned long long strides[2] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.R * i.S * i.c_pad * 2};
+            const unsigned box[3] = {64, 1, (unsigned)t.FT};
+            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_b, w, 3, dims, strides, box);
+            if (s != CPRUNE_OK) return s;
+            plan->map_w = w;
+        }
+        if (plan->map_y != y) {
+            // output [N][P][Q][k_pad]; a store is 64 filters x Wp pixels x TH rows (see the epilogue).  With a fused
+            // pool the kernel stores by hand and the map is not used.
+            const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)i.out_w, (unsigned long long)i.out_h,
+                                                (unsigned long long)i.N};
+            const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)i.out_w * i.k_pad * 2,
+                                                   (unsigned long long)i.out_h * i.out_w * i.k_pad * 2};
+            const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
+            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_y, y, 4, dims, strides, box, false);
+            if (s != CPRUNE_OK) return s;
+            plan->map_y = y;
+        }
+        std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
+        std::memcpy(&tm_w, &plan->tm_b, sizeof(CUtensorMap));
+        std::memcpy(&tm_y, &plan->tm_y, sizeof(CUtensorMap));
+    }
+    static std::mutex attr_mu;
+    static bool attr_set = false;
+    {
+        std::lock_guard<std::mutex> lock(attr_mu);
+        if (!attr_set) {
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            attr_set = true;
+        }
+    }
+    PatchParams p;
+    p.P = i.P; p.Q = i.Q; p.Wp = Wp; p.TH = t.TH; p.tiles_per_img = t.tiles_per_img;
+    p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.FT = t.FT; p.MT = t.MT; p.R = i.R; p.S = i.S; p.pad = i.pad;
+    p.cblks = (i.c_pad + 63) / 64;
+    p.ksteps_last = (i.c_pad - (p.cblks - 1) * 64 + 15) / 16;
+    p.k_pad = i.k_pad;
+    p.act = plan->opts.activation;
+    p.wstages = t.wstages; p.resident = t.resident; p.acc_bufs = t.acc_bufs; p.staging_bufs = t.staging_bufs;
+    p.pool = plan->fused_pool;
+    p.patch_bytes = t.patch_bytes;
+    p.patch_box_bytes = Wp * (t.TH + i.R - 1) * 128;
+    p.bias = b;
+    p.res = (const __nv_bfloat16 *)res;
+    p.y = (__nv_bfloat16 *)y;
+    p.status = device_status_word();
+    if (!p.status) return cuda_fail(cudaGetLastError(), "status word");
+    const int total = i.tiles_m * i.tiles_n;
+    if (total == 0) return CPRUNE_OK;
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    const int grid = total < sms ? total : sms;
+    conv_patch_kernel<<<grid, PK_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, p);
+    CPRUNE_LAUNCH_CHECK("conv_patch_kernel");
+    return CPRUNE_OK;
+}
+
+}  // namespace cprune

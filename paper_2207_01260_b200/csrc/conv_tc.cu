@@ -4,15 +4,17 @@
 //   D[pixel][k] = sum over (r, s, c) of  X[pixel shifted by tap (r,s)][c] * Wt[k][r][s][c]
 //   GEMM-M = N*P*Q output pixels,  GEMM-N = K filters,  GEMM-K = R*S*C
 //
-// One persistent CTA per SM, 192 threads, three roles:
-//   warp 0      producer: per (tap, 64-channel block) one im2col-mode TMA load of PT pixels x 64
+// One persistent CTA per SM, N_PRODUCERS + 9 warps, three roles (warp numbers for N_PRODUCERS = 4; measured: one
+// producer warp is enough for this kernel, which is bound by shared-memory bandwidth):
+//   warps 0..3  producers: per (tap, 64-channel block) one im2col-mode TMA load of PT pixels x 64
 //               channels of the activation tensor (zero fill for the padding border and for
 //               channels beyond c_pad) and one tiled TMA load of FT filters x 64 channels, both
-//               into 128-byte-swizzled shared memory, completion on an mbarrier;
-//   warp 1      one elected lane issues tcgen05.mma (K = 16 per instruction, bf16 x bf16 ->
+//               into 128-byte-swizzled shared memory, completion on an mbarrier; the producer warps
+//               take the pipeline stages in turn;
+//   warp 4      one elected lane issues tcgen05.mma (K = 16 per instruction, bf16 x bf16 ->
 //               float32) with the accumulator in tensor memory; two accumulator buffers so
 //               that the epilogue of one tile overlaps the main loop of the next;
-//   warps 2..5  epilogue: tcgen05.ld the accumulator, bias (+ residual), activation, bf16,
+//   warps 5..12 epilogue: tcgen05.ld the accumulator, bias (+ residual), activation, bf16,
 //               write 64-filter-wide sub-tiles into swizzled shared memory, TMA-store them to
 //               the NHWC output (the store clips rows beyond the last pixel and filters beyond
 //               k_pad by itself).
@@ -32,15 +34,18 @@
 
 #include "common.cuh"
 #include "plan.h"
+#include "sm100_ptx.cuh"
 
 namespace cprune {
 
-constexpr int TC_THREADS = 320;    // producer warp, MMA warp, eight epilogue warps
+constexpr int N_PRODUCERS = 1;     // TMA-issuing warps: pipeline stage i is filled by warp i % N_PRODUCERS
+constexpr int MMA_WARP = N_PRODUCERS;
+constexpr int FIRST_EPI_WARP = N_PRODUCERS + 1;
+constexpr int TC_THREADS = (N_PRODUCERS + 1 + 8) * 32;    // producer warps, MMA warp, eight epilogue warps
 constexpr int BK = 64;             // channels per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;    // column offset of the second accumulator buffer
 constexpr int MAX_STAGES = 8;
-constexpr long long WAIT_LIMIT_CYCLES = 1LL << 31;   // about a second
 constexpr int ORIENT_PIX = 0, ORIENT_FILT = 1;
 constexpr int SUB = 64;            // filters per staged sub-tile (128-byte rows, 128-byte swizzle)
 constexpr int CTRL_BYTES = 2048;   // barriers, flags, bias vector
@@ -70,175 +75,6 @@ struct TcParams {
 // Measured on B200: with kernel parameters beyond 768 bytes (five 128-byte tensor maps + this struct) tasks with
 // many short tiles ran almost twice as slow; the struct therefore has to stay within 128 bytes.
 static_assert(sizeof(TcParams) <= 128, "conv_tc_kernel parameters must stay within 768 bytes");
-
-// ------------------------------------------------------------------------------------------ PTX
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint32_t elect_one() {
-    uint32_t pred = 0;
-    asm volatile(
-        "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
-        "elect.sync rx|px, %1;\n\t"
-        "selp.u32 %0, 1, 0, px;\n\t}"
-        : "=r"(pred)
-        : "r"(0xFFFFFFFFu));
-    return pred;
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-
-// Bounded wait.  Returns false when the limit expired here or (if watch_abort) another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          bool watch_abort = true) {
-    for (int i = 0; i < 64; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    long long t0 = clock64();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (watch_abort && *abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            atomicOr(status, STATUS_TIMEOUT);
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c, int w, int h,
-                                                int n, uint16_t off_w, uint16_t off_h) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-        :
-        : "r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5}], [%2];"
-        :
-        : "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4}], [%2];"
-        :
-        : "r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 :
-                 : "l"(map), "r"(src), "r"(c0), "r"(c1)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void tma_store_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        :
-        : "r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// mbarrier arrives once every tcgen05.mma issued so far by this thread has completed
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t *v) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, 128-byte
-// swizzled, with 8-row groups 1024 bytes apart (the layout both TMA loads produce).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);   // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                  // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                  // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                  // 128-byte swizzle
-    return d;
-}
-
-// Descriptor of a K-major bf16 operand stored without swizzle as 8-row x 16-byte core matrices:
-// rows 16 bytes apart, 8-row groups 128 bytes apart, the next 8 channels `k_stride` bytes away
-// (the layout of one im2col TMA load of 8 channels per pixel; successive taps follow each other).
-__device__ __forceinline__ uint64_t smem_desc_interleaved(uint32_t addr, uint32_t k_stride) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((k_stride >> 4) & 0x3FFF) << 16;   // leading byte offset: next core matrix along K
-    d |= (uint64_t)(128 >> 4) << 32;                   // stride byte offset: next 8 rows
-    d |= (uint64_t)1 << 46;
-    return d;
-}
-
-// Descriptor of a K-major bf16 operand whose rows are 32 bytes (16 channels), 32-byte swizzled, 8-row groups
-// 256 bytes apart: one im2col load of 16 channels per (paired) pixel = exactly one K = 16 step.
-__device__ __forceinline__ uint64_t smem_desc_sw32(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(256 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)6 << 61;                  // 32-byte swizzle
-    return d;
-}
-
-// Byte offset of (row, 16-byte chunk c of 8) in a staged sub-tile of 128-byte rows under the
-// 128-byte swizzle (address bits 4..6 are XORed with bits 7..9, i.e. with the row modulo 8).
-__device__ __forceinline__ uint32_t sub_off(int row, int c) { return (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)); }
 
 // 2x2 stride-2 max-pool of NPX consecutive pixels (whole row pairs of Q pixels, Q a power of two) held by
 // one thread for one filter: NPX / 4 pooled values, written to rows t0.. of a staged sub-tile.
@@ -283,7 +119,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     uint32_t *tmem_slot = (uint32_t *)(ctrl + 8 * (2 * MAX_STAGES + 5));
     volatile int *abort_flag = (volatile int *)(ctrl + 8 * (2 * MAX_STAGES + 5) + 4);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the shuffle tells the compiler that the warp number is the same in all lanes, so that the role code below
+    // (loop counters, descriptors, TMA coordinates) can live in uniform registers
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -298,7 +136,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
@@ -311,9 +149,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     const int total_tiles = p.tiles_m * p.tiles_n * p.splits;   // work items: (tile, K slice), slice fastest
     const int PQ = p.P * p.Q;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ producer
-        int stage = 0;
+    if (warp < N_PRODUCERS) {
+        // ------------------------------------------------------------------ producers
+        // Issuing one TMA load costs the issuing thread about 300 cycles whatever the box size (measured), so
+        // one warp cannot feed the tensor core.  Every producer warp walks the same sequence of pipeline
+        // stages and fills those whose running index is congruent to its warp number.
+        int stage = 0, turn = 0;
         uint32_t phase = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total_tiles && ok; item += gridDim.x) {
@@ -343,9 +184,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 const int taps = p.R * p.pair_taps;
                 const int wcp = q0 - ((p.pad + 1) >> 1);
                 for (int it = 0; it < p.iters - p.res_iters; ++it) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                    const bool mine = turn == warp;
+                    if (++turn == N_PRODUCERS) turn = 0;
+                    if (mine) ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                     if (!ok) break;
-                    if (elect_one()) {
+                    if (mine && elect_one()) {
                         const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
                         int loads = taps - it * 4;
                         if (loads > 4) loads = 4;
@@ -365,9 +208,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 // 8 taps x 8 channels per stage; every tap is its own im2col load of PT pixels x 16 bytes
                 const int taps = p.R * p.S;
                 for (int it = 0; it < p.iters - p.res_iters; ++it) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                    const bool mine = turn == warp;
+                    if (++turn == N_PRODUCERS) turn = 0;
+                    if (mine) ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                     if (!ok) break;
-                    if (elect_one()) {
+                    if (mine && elect_one()) {
                         const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
                         int nt = taps - it * 8;
                         if (nt > 8) nt = 8;
@@ -396,9 +241,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             const int it_last = it_end - (p.splits == 1 ? p.res_iters : 0);
             const int k0 = nt_f * p.FT;
             for (int it = it_begin; it < it_last; ++it) {
-                ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                const bool mine = turn == warp;
+                if (++turn == N_PRODUCERS) turn = 0;
+                if (mine) ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                 if (!ok) break;
-                if (elect_one()) {
+                if (mine && elect_one()) {
                     const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
                     const uint32_t fb = full_bar(stage);
                     mbar_expect_tx(fb, (uint32_t)stage_bytes);
@@ -417,9 +264,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
             // operand and a 64-column slice of the identity matrix the filter-side operand, so that the
             // MMA adds residual[pixel][k] to accumulator row k
             for (int j = 0; j < p.res_iters && ok; ++j) {
-                ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
+                const bool mine = turn == warp;
+                if (++turn == N_PRODUCERS) turn = 0;
+                if (mine) ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status));
                 if (!ok) break;
-                if (elect_one()) {
+                if (mine && elect_one()) {
                     const uint32_t x_dst = base + (uint32_t)stage * stage_bytes;
                     mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
                     tma_load_2d(x_dst, &tm_res, full_bar(stage), j * BK, (int)m0);
@@ -429,7 +278,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                 if (++stage == p.stages) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == MMA_WARP) {
         // ------------------------------------------------------------------ MMA issue
         // instruction descriptor: D float32, A and B bf16, both K-major, M = 128, N = filters or pixels
         const int mma_n = ORIENT == ORIENT_PIX ? p.FT : p.PT;
@@ -537,9 +386,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
         // Two warps share each quarter of the tensor-memory lanes (a warp may only read lanes 32*(warp%4)..+31):
         // `half` says which half of every group's columns this warp takes.
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - FIRST_EPI_WARP) >> 2;
         const int trow = quarter * 32 + lane;          // accumulator row (pixel or filter) of this thread
-        const bool store_thread = warp == 2 && lane == 0;
+        const bool store_thread = warp == FIRST_EPI_WARP && lane == 0;
         int acc = 0;
         uint32_t acc_phase = 0, epi_phase = 0;
         uint32_t group_counter = 0;                    // staged groups so far (selects the buffer)
@@ -776,7 +625,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
@@ -900,6 +749,22 @@ cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, con
     return CPRUNE_OK;
 }
 
+cprune_status encode_tiled_bf16_sw128(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
+                                      const unsigned long long *strides_bytes, const unsigned *box, bool for_loads) {
+    cprune_status st = load_driver_entry_points();
+    if (st != CPRUNE_OK) return st;
+    cuuint64_t d[5], s[4];
+    cuuint32_t b[5], e[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; e[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
+    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(ptr), d, s, b, e,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                for_loads ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(swizzle 128)");
+    return CPRUNE_OK;
+}
+
 static int smem_for(int stages, int PT, int FT, int staging_bufs, int group_rows) {
     (void)group_rows;
     return 1024 /* alignment slack */ + stages * (PT + FT) * BK * 2 + staging_bufs * GROUP_BYTES + CTRL_BYTES;
@@ -909,6 +774,10 @@ static int smem_for(int stages, int PT, int FT, int staging_bufs, int group_rows
 cprune_status plan_conv_tensor(cprune_plan *plan) {
     cprune_plan_info &i = plan->info;
     if (i.groups != 1) return CPRUNE_ERR_UNSUPPORTED;
+    // stride-1 tasks with more than one tap: patch kernel when its tile is well filled
+    plan->patch = 0;
+    const char *no_patch = getenv("CPRUNE_NO_PATCH");      // measurement override
+    if (!(no_patch && no_patch[0] == '1') && plan_conv_patch(plan) == CPRUNE_OK) return CPRUNE_OK;
     if (i.R > 16 || i.S > 16 || i.pad > 64 || i.stride > 8) return CPRUNE_ERR_UNSUPPORTED;
     if (i.W > 65535 || i.H > 65535) return CPRUNE_ERR_UNSUPPORTED;
     const long long M = (long long)i.N * i.P * i.Q;
@@ -1108,6 +977,7 @@ static int sm_count() {
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
                                  void *y, void *partial, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
+    if (plan->patch) return launch_conv_patch(plan, x, w, b, res, y, st);
     CUtensorMap tm_x, tm_w, tm_y, tm_res, tm_id;
     const bool split = plan->splits > 1;
     if (split && !partial) return CPRUNE_ERR_INVALID_ARG;

@@ -9,6 +9,12 @@
 
 #include "cprune.h"
 
+// Tiling of the patch kernel (conv_patch.cu): a tile is TH output rows of one image, MT blocks of 128 accumulator
+// rows, FT filters.
+struct PatchTiling {
+    int MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes;
+};
+
 struct cprune_plan {
     cprune_plan_info info;
     cprune_task_opts opts;
@@ -35,6 +41,8 @@ struct cprune_plan {
     size_t partial_bytes = 0;       // float32 partial sums in the workspace
     int small_c = 0;                // 3-channel stems: 1 = 8 taps x 8 channels per K block, 2 = pixel pairs
     int s_packed = 0;               // filter taps per row in the packed weights (S, or S + 1 in pair mode)
+    int patch = 0;                  // 1: stride-1 task on the patch kernel (conv_patch.cu)
+    PatchTiling pt = {};
 };
 
 namespace cprune {
@@ -49,6 +57,13 @@ cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, 
 cprune_status plan_conv_tensor(cprune_plan *plan);  // fills tile fields of plan->info; UNSUPPORTED if not eligible
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
                                  void *y, void *partial, cudaStream_t st);
+// stride-1 R x S > 1 tasks with the input patch resident in shared memory (part of the tensor family)
+cprune_status plan_conv_patch(cprune_plan *plan);   // UNSUPPORTED if the task is not eligible or would waste the tile
+cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
+                                void *y, cudaStream_t st);
+// tiled bf16 tensor map with the 128-byte swizzle (inner box extent 64 elements), out-of-bounds elements read as zero
+cprune_status encode_tiled_bf16_sw128(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
+                                      const unsigned long long *strides_bytes, const unsigned *box, bool for_loads = true);
 // tiled bf16 tensor map without swizzle, out-of-bounds elements read as zero
 cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
                                 const unsigned long long *strides_bytes, const unsigned *box);
