@@ -105,7 +105,7 @@ __device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint32_t FT, uint32_t
 
 __global__ void __launch_bounds__(PK_THREADS, 1)
 conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                  const __grid_constant__ CUtensorMap tm_y, const PatchParams p) {
+                  const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res, const PatchParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -122,6 +122,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     auto tfull = [&](int a) { return ctrl0 + 32u + 8u * a; };
     auto tempty = [&](int a) { return ctrl0 + 48u + 8u * a; };
     const uint32_t epi_bar = ctrl0 + 64u;
+    auto res_full = [&](int b) { return ctrl0 + 80u + 8u * b; };   // residual tile landed in staging buffer b
     uint32_t *tmem_slot = (uint32_t *)(ctrl + 72);
     volatile int *abort_flag = (volatile int *)(ctrl + 76);
     auto wfull = [&](int s) { return ctrl0 + 128u + 8u * s; };
@@ -139,6 +140,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         for (int a = 0; a < 2; ++a) { mbar_init(tfull(a), p.MT); mbar_init(tempty(a), 8); }
         for (int s = 0; s < p.wstages; ++s) { mbar_init(wfull(s), 1); mbar_init(wempty(s), p.MT); }
         mbar_init(epi_bar, 8);
+        mbar_init(res_full(0), 1);
+        mbar_init(res_full(1), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -282,14 +285,25 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             epi_phase ^= 1u;
             return r;
         };
-        // this thread's slot in each accumulator block never changes: where its pixel goes (elements from the tile's
-        // first pixel) and which tile row it is in; x < 0: a wrap-around or unused slot
-        const int2 my_slot[2] = {lut[trow], lut[128 + trow]};
         // activation as a clamp: no branches in the per-element code
         const float act_lo = p.act == CPRUNE_ACT_NONE ? -INFINITY : 0.f, act_hi = p.act == CPRUNE_ACT_RELU6 ? 6.f : INFINITY;
         const bool store_thread = warp == PK_FIRST_EPI && lane == 0;
         const int groups = (p.FT + 63) / 64;
         const int n_entries = p.pool ? (p.TH >> 1) * (p.Q >> 1) : 128 * p.MT;
+        // The residual of a group arrives by TMA in the staging buffer the group will use (same box as the store:
+        // wrap-around slots read as zero); the values are added there in place.  The load for the next group is
+        // issued as soon as its buffer is free.
+        const bool with_res = p.res != nullptr;
+        auto load_residual = [&](int item_, int g_, uint32_t counter) {
+            int tm_ = item_, nt_ = 0;
+            if (p.tiles_n > 1) { tm_ = item_ / p.tiles_n; nt_ = item_ - tm_ * p.tiles_n; }
+            const int n_ = tm_ / p.tiles_per_img;
+            const int p0_ = (tm_ - n_ * p.tiles_per_img) * p.TH;
+            const uint32_t b = p.staging_bufs == 2 ? (counter & 1u) : 0u;
+            mbar_expect_tx(res_full(b), (uint32_t)(p.TH * p.Wp * 128));
+            tma_load_4d(staging0 + b * stage_buf_bytes, &tm_res, res_full(b), nt_ * p.FT + g_ * 64, 0, p0_, n_);
+        };
+        if (with_res && store_thread && (int)blockIdx.x < total_items) load_residual(blockIdx.x, 0, 0);
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
             int tm = item, nt = 0;
             if (p.tiles_n > 1) { tm = item / p.tiles_n; nt = item - tm * p.tiles_n; }
@@ -307,6 +321,12 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 const uint32_t boff = (p.staging_bufs == 2 ? (group_counter & 1u) : 0u) * stage_buf_bytes;
                 uint8_t *buf = smem + (staging0 - base) + boff;
                 const int ch = g * 64 + half * 32;           // this warp's 32 filters of the group
+                if (with_res) {
+                    const uint32_t b = p.staging_bufs == 2 ? (group_counter & 1u) : 0u;
+                    const uint32_t par = p.staging_bufs == 2 ? ((group_counter >> 1) & 1u) : (group_counter & 1u);
+                    ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), par, abort_flag, p.status, false));
+                    if (!ok) break;
+                }
                 for (int mb = 0; mb < p.MT; ++mb) {
                     const int slot = mb * 128 + trow;
                     uint32_t v[32];
@@ -314,14 +334,10 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     for (int sb = 0; sb < 2; ++sb)
                         if (ch + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(mb * p.FT + ch + sb * 16), v + sb * 16);
                     bf16x8 rv[4];
-                    const int2 ms = my_slot[mb];
-                    const bool px_ok = !p.pool && ms.x >= 0 && (ms.x >> 16) < rows_valid;
-                    const bool has_res = p.res != nullptr && px_ok;
-                    if (has_res) {
-                        const __nv_bfloat16 *rrow = p.res + in_tile + ms.y + k0 + ch;
+                    if (with_res) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
-                            if (k0 + ch + j * 8 < p.k_pad) rv[j] = ldg8((const bf16x8 *)(rrow + j * 8));
+                            rv[j] = *(const bf16x8 *)(buf + mb * PK_BLOCK_BYTES + sub_off(trow, half * 4 + j));
                     }
                     tmem_ld_wait();
                     if (g == groups - 1 && mb == p.MT - 1) {     // accumulator fully read: hand it back
@@ -341,7 +357,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                                 const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[sb * 16 + h * 8 + j]) + bb[j];
-                                if (has_res && k0 + c0 + h * 8 < p.k_pad) {
+                                if (with_res) {
                                     float rf[8];
                                     unpack8(rv[sb * 2 + h], rf);
 #pragma unroll
@@ -367,6 +383,13 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                         if (k0 + g * 64 < p.k_pad) tma_store_4d(&tm_y, staging0 + boff, k0 + g * 64, 0, p0, n);
                         tma_store_commit();
                         if (p.staging_bufs == 1) tma_store_wait_read<0>();
+                        if (with_res) {
+                            // next group of this CTA: its buffer is free (two buffers: its last store was waited for
+                            // before the barrier above; one buffer: just now)
+                            int ni = item, ng = g + 1;
+                            if (ng == groups) { ni = item + gridDim.x; ng = 0; }
+                            if (ni < total_items) load_residual(ni, ng, group_counter + 1);
+                        }
                     }
                     if (p.staging_bufs == 1) {
                         ok = epi_sync();
@@ -530,7 +553,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     const cprune_plan_info &i = plan->info;
     const PatchTiling &t = plan->pt;
     const int Wp = i.W + 2 * i.pad;
-    CUtensorMap tm_x, tm_w, tm_y;
+    CUtensorMap tm_x, tm_w, tm_y, tm_res;
     {
         std::lock_guard<std::mutex> lock(plan->mu);
         if (plan->map_x != x) {
@@ -565,7 +588,18 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
         }
         std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
         std::memcpy(&tm_w, &plan->tm_b, sizeof(CUtensorMap));
+        if (res && plan->map_res != res) {
+            const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)i.Q, (unsigned long long)i.P,
+                                                (unsigned long long)i.N};
+            const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)i.Q * i.k_pad * 2,
+                                                   (unsigned long long)i.P * i.Q * i.k_pad * 2};
+            const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
+            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_res, res, 4, dims, strides, box);
+            if (s != CPRUNE_OK) return s;
+            plan->map_res = res;
+        }
         std::memcpy(&tm_y, &plan->tm_y, sizeof(CUtensorMap));
+        std::memcpy(&tm_res, res ? &plan->tm_res : &plan->tm_y, sizeof(CUtensorMap));
     }
     static std::mutex attr_mu;
     static bool attr_set = false;
@@ -598,7 +632,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
     const int grid = total < sms ? total : sms;
-    conv_patch_kernel<<<grid, PK_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, p);
+    conv_patch_kernel<<<grid, PK_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, p);
     CPRUNE_LAUNCH_CHECK("conv_patch_kernel");
     return CPRUNE_OK;
 }
