@@ -50,10 +50,12 @@ constexpr int PK_BLOCK_BYTES = 16384;    // staged block: 128 slots x 64 filters
 
 struct PatchParams {
     int P, Q, Wp, TH, tiles_per_img, tiles_m, tiles_n;
-    int FT, MT, R, S, pad, cblks, ksteps_last, k_pad;
+    int FT, MT, R, S, pad, pad_w, cblks, ksteps_last, k_pad;   // pad: rows above the image in a patch; pad_w: columns left of it
     int act, wstages, resident, acc_bufs, staging_bufs, pool;
     int patch_bytes;       // shared memory of one patch stage
     int patch_box_bytes;   // bytes one patch load delivers
+    int w_stage_bytes;     // shared memory of one filter stage (FT rows, rounded up to 1024 bytes)
+    int rb16;              // bytes per pixel row in shared memory / 16: 8 (64 channels) or 2 (16 channels, regrouped stems)
     const float *bias;
     const __nv_bfloat16 *res;
     __nv_bfloat16 *y;
@@ -69,33 +71,23 @@ __device__ __forceinline__ uint4 bf16x8_max(uint4 a, uint4 b) {
     return r;
 }
 
-// All MMAs of one filter tap: for each of the MT accumulator blocks, nk steps of 16 channels.  a_lo and w_lo are
+// All MMAs of one filter tap for one accumulator block: nk steps of 16 channels.  a_lo and w_lo are
 // the low words of the operand descriptors (start address in 16-byte units).  Called by the whole warp: the
 // operands are computed by all lanes (they stay in uniform registers) and one elected lane issues.
-template <int MT>
-__device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint32_t FT, uint32_t a_lo, uint32_t w_lo, uint32_t idesc,
+__device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint32_t a_lo, uint32_t w_lo, uint32_t desc_hi, uint32_t idesc,
                                           uint32_t accumulate, int nk, uint32_t commit_w, uint32_t commit_p) {
-    uint32_t al[MT][4], wl[4], dd[MT];
+    uint32_t al[4], wl[4];
 #pragma unroll
-    for (int kk = 0; kk < 4; ++kk) wl[kk] = w_lo + (uint32_t)(2 * kk);
-#pragma unroll
-    for (int mb = 0; mb < MT; ++mb) {
-        dd[mb] = d_tmem + (uint32_t)mb * FT;
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) al[mb][kk] = a_lo + (uint32_t)(mb * 1024 + 2 * kk);
-    }
+    for (int kk = 0; kk < 4; ++kk) { wl[kk] = w_lo + (uint32_t)(2 * kk); al[kk] = a_lo + (uint32_t)(2 * kk); }
     if (elect_one()) {
         if (nk == 4) {
 #pragma unroll
-            for (int mb = 0; mb < MT; ++mb)
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16_sw128(dd[mb], al[mb][kk], wl[kk], idesc, kk ? 1u : accumulate);
+            for (int kk = 0; kk < 4; ++kk) umma_bf16_words(d_tmem, al[kk], wl[kk], desc_hi, idesc, kk ? 1u : accumulate);
         } else {
+            umma_bf16_words(d_tmem, al[0], wl[0], desc_hi, idesc, accumulate);
 #pragma unroll
-            for (int mb = 0; mb < MT; ++mb)
-#pragma unroll
-                for (int kk = 0; kk < 3; ++kk)
-                    if (kk < nk) umma_bf16_sw128(dd[mb], al[mb][kk], wl[kk], idesc, kk ? 1u : accumulate);
+            for (int kk = 1; kk < 3; ++kk)
+                if (kk < nk) umma_bf16_words(d_tmem, al[kk], wl[kk], desc_hi, idesc, 1u);
         }
         if (commit_w) umma_commit(commit_w);
         if (commit_p) umma_commit(commit_p);
@@ -110,7 +102,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - raw);
-    const uint32_t w_bytes = (uint32_t)p.FT * 128u;
+    const uint32_t w_bytes = (uint32_t)p.w_stage_bytes;                   // stage stride
+    const uint32_t w_tx_bytes = (uint32_t)p.FT * 16u * (uint32_t)p.rb16;  // bytes one filter load delivers
     const uint32_t patch0 = base;
     const uint32_t w0 = patch0 + PK_PATCH_STAGES * (uint32_t)p.patch_bytes;
     const uint32_t staging0 = w0 + (uint32_t)p.wstages * w_bytes;
@@ -183,7 +176,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (!ok) break;
                 if (elect_one()) {
                     mbar_expect_tx(pfull(ps), (uint32_t)p.patch_box_bytes);
-                    tma_load_4d(patch0 + (uint32_t)ps * p.patch_bytes, &tm_x, pfull(ps), cb * 64, -p.pad, p0 - p.pad, n);
+                    tma_load_4d(patch0 + (uint32_t)ps * p.patch_bytes, &tm_x, pfull(ps), cb * 64, -p.pad_w, p0 - p.pad, n);
                 }
                 __syncwarp();
                 if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; }
@@ -208,7 +201,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                         if (!p.resident) ok = __all_sync(0xffffffffu, mbar_wait(wempty(ws), wphase ^ 1u, abort_flag, p.status));
                         if (!ok) break;
                         if (elect_one()) {
-                            mbar_expect_tx(wfull(ws), w_bytes);
+                            mbar_expect_tx(wfull(ws), w_tx_bytes);
                             tma_load_3d(w0 + (uint32_t)ws * w_bytes, &tm_w, wfull(ws), cb * 64, tap, k0);
                         }
                         __syncwarp();
@@ -230,9 +223,11 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         bool ok = true;
         // A lone warp pays several cycles for every instruction, so the loop works on the low descriptor words
         // only (32-bit adds) and issues a tap's MMAs from fully unrolled code.
-        const uint32_t patch_lo0 = desc_lo_sw128(patch0), w_lo0 = desc_lo_sw128(w0);
+        const uint32_t patch_lo0 = desc_lo(patch0), w_lo0 = desc_lo(w0);
+        const uint32_t desc_hi = p.rb16 == 8 ? DESC_HI_SW128 : DESC_HI_SW32;
+        const uint32_t slot_step = (uint32_t)p.rb16;                    // descriptor units (16 bytes) per pixel row
         const uint32_t patch_step = (uint32_t)p.patch_bytes >> 4, w_step = w_bytes >> 4;
-        const uint32_t row_step = (uint32_t)((p.Wp - p.S + 1) * 8);   // descriptor units (16 bytes) from tap (r, S-1) to (r+1, 0)
+        const uint32_t row_step = (uint32_t)(p.Wp - p.S + 1) * slot_step;   // from tap (r, S-1) to (r+1, 0)
         uint32_t patch_lo = patch_lo0, w_lo = w_lo0;
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
             ok = __all_sync(0xffffffffu, mbar_wait(tempty(acc), acc_phase ^ 1u, abort_flag, p.status));
@@ -244,7 +239,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 ok = __all_sync(0xffffffffu, mbar_wait(pfull(ps), pphase, abort_flag, p.status));
                 if (!ok) break;
                 const int nk = cb == p.cblks - 1 ? p.ksteps_last : 4;
-                uint32_t tap_lo = patch_lo + (uint32_t)(mb * 1024);      // the second block's slots start 16 KB further on
+                uint32_t tap_lo = patch_lo + (uint32_t)(mb * 128) * slot_step;      // the second block's slots follow the first's
                 int s = 0;
                 for (int tap = 0; tap < RS; ++tap) {
                     // resident filters: the barrier completes once (first tile) and stays complete for parity 0
@@ -252,13 +247,13 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     if (!ok) break;
                     {
                         const uint32_t cw = p.resident ? 0u : wempty(ws), cp = tap == RS - 1 ? pempty(ps) : 0u;
-                        issue_tap<1>(d_tmem, (uint32_t)p.FT, tap_lo, w_lo, idesc, accumulate, nk, cw, cp);
+                        issue_tap(d_tmem, tap_lo, w_lo, desc_hi, idesc, accumulate, nk, cw, cp);
                     }
                     accumulate = 1;
                     w_lo += w_step;
                     if (++ws == p.wstages) { ws = 0; wphase ^= 1u; w_lo = w_lo0; }
-                    tap_lo += 8;
-                    if (++s == p.S) { s = 0; tap_lo += row_step - 8; }
+                    tap_lo += slot_step;
+                    if (++s == p.S) { s = 0; tap_lo += row_step - slot_step; }
                 }
                 patch_lo += patch_step;
                 if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; patch_lo = patch_lo0; }
@@ -442,33 +437,76 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 // Estimated cycles of one tile.  Per tcgen05.mma (M = 128, N = FT, K = 16) the tensor pipe needs FT / 2 cycles
 // and the operand reads (128 + FT) * 32 bytes of the 128 bytes per clock that shared memory delivers; the TMA
 // writes of filters and patches share that port (measured on B200).
-static double tile_cycles(int MT, int FT, int RS, int cblks, int ksteps_last, int Wp, int TH, int R, bool resident,
+static double tile_cycles(int MT, int FT, int RS, int cblks, int ksteps_last, int row_bytes, int Wp, int TH, int R, bool resident,
                           int acc_bufs) {
     double total = 0;
     for (int cb = 0; cb < cblks; ++cb) {
         const int nk = cb == cblks - 1 ? ksteps_last : 4;
         const double tensor = MT * nk * (FT / 2.0);
-        const double smem = (MT * nk * (128.0 + FT) * 32.0 + (resident ? 0.0 : FT * 128.0)) / 128.0;
-        total += RS * (tensor > smem ? tensor : smem) + Wp * (TH + R - 1);
+        const double smem = (MT * nk * (128.0 + FT) * 32.0 + (resident ? 0.0 : FT * (double)row_bytes)) / 128.0;
+        total += RS * (tensor > smem ? tensor : smem) + Wp * (TH + R - 1) * row_bytes / 128.0;
     }
-    const double epilogue = MT * ((FT + 63) / 64) * 500.0;
+    const double epilogue = MT * ((FT + 63) / 64) * 1200.0;
     return total + (acc_bufs == 2 ? (epilogue > total ? epilogue - total : 0.0) : epilogue) + 1500.0;
+}
+
+// What the kernel sees.  Wide tasks (c_pad >= 16, stride 1): the task itself, 64 channels per shared-memory row.
+// Stems with C * stride^2 <= 16 (stride 1 or 2): the input is first regrouped into 16-channel pixels, one per
+// stride x stride block of input pixels (channel (dy * stride + dx) * C + c), with the zero columns of the padding
+// written out.  Up to four consecutive regrouped pixels (the Se filter columns, 32 bytes each) are then read as
+// ONE 128-byte shared-memory row through a tensor map whose pixel stride is 32 bytes, so that the task becomes a
+// stride-1 task with Re x 1 taps of Se * 16 channels and no wrap-around slots.  (Rows of 32 bytes would work too,
+// but the MMA's operand reads then cost a full shared-memory cycle per row: measured four times slower.)
+struct PatchGeometry {
+    int stem, sf, Re, Se, pad_lo, He, We, WP, cblks, ksteps_last, Wp, kR, kS, pad_w;
+};
+
+static bool patch_geometry(const cprune_plan_info &i, PatchGeometry *g) {
+    if (i.groups != 1) return false;
+    if (i.c_pad >= 16 && i.stride == 1) {
+        if (i.R * i.S <= 1 || i.R > 7 || i.S > 7) return false;
+        g->stem = 0; g->sf = 1; g->Re = i.R; g->Se = i.S; g->pad_lo = i.pad; g->He = i.H; g->We = i.W; g->WP = i.W;
+        g->cblks = (i.c_pad + 63) / 64;
+        g->ksteps_last = (i.c_pad - (g->cblks - 1) * 64 + 15) / 16;
+        g->Wp = i.Q + i.S - 1;
+        g->kR = i.R; g->kS = i.S; g->pad_w = i.pad;
+        if (g->Wp < g->We + g->pad_lo) return false;
+    } else if (i.c_pad == 8 && i.stride <= 2 && i.C * i.stride * i.stride <= 16 && i.R * i.S > 1 && i.R <= 8 && i.S <= 8) {
+        const int sf = i.stride;
+        if ((i.H % sf) || (i.W % sf)) return false;
+        if (i.R - 1 - i.pad < 0 || i.S - 1 - i.pad < 0) return false;
+        g->stem = 1; g->sf = sf;
+        g->pad_lo = sf == 1 ? i.pad : (i.pad + 1) / 2;
+        g->Re = sf == 1 ? i.R : (i.R - 1 - i.pad) / 2 + g->pad_lo + 1;
+        g->Se = sf == 1 ? i.S : (i.S - 1 - i.pad) / 2 + g->pad_lo + 1;
+        if (g->Se > 4) return false;
+        g->He = i.H / sf; g->We = i.W / sf;
+        g->WP = i.Q + 3;                       // a row starting at the last output column still reads four pixels
+        if (g->WP < g->We + g->pad_lo) return false;
+        g->cblks = 1; g->ksteps_last = g->Se;
+        g->Wp = i.Q;
+        g->kR = g->Re; g->kS = 1; g->pad_w = 0;
+    } else {
+        return false;
+    }
+    if (g->Wp > 128) return false;
+    if (i.P + g->Re - 1 < g->He + g->pad_lo) return false;
+    return true;
 }
 
 // Decides whether the task runs on the patch kernel and with which tiling; fills plan->info tile fields.
 cprune_status plan_conv_patch(cprune_plan *plan) {
     cprune_plan_info &i = plan->info;
     plan->patch = 0;
-    if (i.groups != 1 || i.stride != 1 || i.R * i.S <= 1 || i.R > 7 || i.S > 7) return CPRUNE_ERR_UNSUPPORTED;
-    if (i.c_pad < 16) return CPRUNE_ERR_UNSUPPORTED;
-    const int Wp = i.W + 2 * i.pad;
-    if (Wp > 128 || i.Q != Wp - i.S + 1 || i.H + 2 * i.pad - i.R + 1 != i.P) return CPRUNE_ERR_UNSUPPORTED;
+    plan->pre_bytes = 0;
+    PatchGeometry g;
+    if (!patch_geometry(i, &g)) return CPRUNE_ERR_UNSUPPORTED;
+    const int Wp = g.Wp;
     const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
     if (pool && (plan->opts.residual || (i.P & 1) || (i.Q & 1))) return CPRUNE_ERR_UNSUPPORTED;
     const int k16 = round_up(i.K, 16);
-    const int cblks = (i.c_pad + 63) / 64;
-    const int ksteps_last = (i.c_pad - (cblks - 1) * 64 + 15) / 16;
-    const int RS = i.R * i.S;
+    const int cblks = g.cblks, ksteps_last = g.ksteps_last, RB = 128;
+    const int RS = g.kR * g.kS;
     double best = 1e30;
     PatchTiling bt = {};
     const char *force_mt = getenv("CPRUNE_PATCH_MT");       // measurement overrides
@@ -488,30 +526,31 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             if (FT > 256 || MT * FT > 512) continue;
             if ((k16 + FT - 1) / FT != tiles_n) continue;
             const int acc_bufs = 2 * MT * FT <= 512 ? 2 : 1;
-            const int patch_bytes = round_up((128 * MT + (i.R - 1) * Wp + i.S - 1) * 128, 1024);
-            if (patch_bytes < Wp * (TH + i.R - 1) * 128) continue;
+            const int patch_bytes = round_up((128 * MT + (g.kR - 1) * Wp + g.kS - 1) * RB, 1024);
+            if (patch_bytes < Wp * (TH + g.kR - 1) * RB) continue;
             const int fixed = 1024 + PK_PATCH_STAGES * patch_bytes + PK_CTRL_BYTES;
             const int budget = 227 * 1024 - fixed;
             const int sb_max = 2, sb_min = 1;
+            const int w_stage = round_up(FT * RB, 1024);
             int staging_bufs = sb_max, wstages = 0, resident = 0;
             // resident filters when the whole set of this filter tile fits
             if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES) {
                 for (int sb = sb_max; sb >= sb_min && !resident; --sb)
-                    if (RS * cblks * FT * 128 + sb * MT * PK_BLOCK_BYTES <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
+                    if (RS * cblks * w_stage + sb * MT * PK_BLOCK_BYTES <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
             }
             if (!resident) {
                 staging_bufs = sb_max;
-                wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / (FT * 128);
+                wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / w_stage;
                 if (wstages < 3 && sb_min < sb_max) {
                     staging_bufs = sb_min;
-                    wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / (FT * 128);
+                    wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / w_stage;
                 }
                 if (wstages < 3) continue;
                 if (wstages > 8) wstages = 8;
             }
             const long long tiles = (long long)i.N * tiles_per_img * tiles_n;
             const double waves = (double)((tiles + 147) / 148);
-            double t = waves * tile_cycles(MT, FT, RS, cblks, ksteps_last, Wp, TH, i.R, resident != 0, acc_bufs);
+            double t = waves * tile_cycles(MT, FT, RS, cblks, ksteps_last, RB, Wp, TH, g.kR, resident != 0, acc_bufs);
             if (resident) t += RS * cblks * FT;    // one-time filter load
             if (t < best) {
                 best = t;
@@ -527,12 +566,14 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     if ((long long)i.N * bt.tiles_per_img * bt.tiles_n < 64) return CPRUNE_ERR_UNSUPPORTED;
     plan->patch = 1;
     plan->pt = bt;
+    plan->narrow = g.stem;
     plan->orient = 0;
     plan->small_c = 0;
     plan->s_packed = i.S;
     plan->splits = 1;
     plan->ipp = 0;
     plan->partial_bytes = 0;
+    plan->pre_bytes = g.stem ? ((size_t)i.N * g.He * g.WP * 32 + 255) / 256 * 256 : 0;
     plan->fused_pool = pool ? 1 : 0;
     i.tile_m = 128 * bt.MT;
     i.tile_n = bt.FT;
@@ -543,34 +584,129 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     i.k_alloc = bt.tiles_n * bt.FT;
     const int ksteps = (cblks - 1) * 4 + ksteps_last;
     i.padded_flops = 2.0 * (double)i.tiles_m * i.tile_m * (double)i.k_alloc * RS * ksteps * 16.0;
-    plan->smem_bytes = 1024 + PK_PATCH_STAGES * bt.patch_bytes + bt.wstages * bt.FT * 128 + bt.staging_bufs * bt.MT * PK_BLOCK_BYTES +
-                       PK_CTRL_BYTES;
+    plan->smem_bytes = 1024 + PK_PATCH_STAGES * bt.patch_bytes + bt.wstages * round_up(bt.FT * RB, 1024) +
+                       bt.staging_bufs * bt.MT * PK_BLOCK_BYTES + PK_CTRL_BYTES;
     return CPRUNE_OK;
 }
 
+// Regroups a bf16 NHWC tensor with c_pad = 8 channels (C real ones) into 16-channel pixels, one per sf x sf block of
+// input pixels, in rows of WP pixels of which the first pad_lo (and whatever follows the image) are zero:
+// out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
+__global__ void __launch_bounds__(256) regroup_kernel(const bf16x8 *__restrict__ x, int N, int H, int W, int C, int sf, int pad_lo,
+                                                      int WP, uint4 *__restrict__ out) {
+    const int H2 = H / sf, W2 = W / sf;
+    const long long total = (long long)N * H2 * WP;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        const int wp = (int)(e % WP);
+        const long long t = e / WP;
+        const int h2 = (int)(t % H2);
+        const long long n = t / H2;
+        const int w2 = wp - pad_lo;
+        __align__(16) __nv_bfloat16 o[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) o[c] = __float2bfloat16_rn(0.f);
+        if (w2 >= 0 && w2 < W2) {
+            for (int dy = 0; dy < sf; ++dy)
+                for (int dx = 0; dx < sf; ++dx) {
+                    const bf16x8 v = ldg8(x + (n * H + sf * h2 + dy) * W + sf * w2 + dx);
+                    const __nv_bfloat16 *pv = reinterpret_cast<const __nv_bfloat16 *>(&v);
+                    for (int c = 0; c < C; ++c) o[(dy * sf + dx) * C + c] = pv[c];
+                }
+        }
+        out[2 * e] = *reinterpret_cast<const uint4 *>(o);
+        out[2 * e + 1] = *reinterpret_cast<const uint4 *>(o + 8);
+    }
+}
+
+// Filters of a regrouped stem: out[k][re * Se + se][(dy * sf + dx) * C + c] = w[k][c][sf * re + dy - er][sf * se + dx - es]
+// (zero where that tap does not exist), er = sf * pad_lo - pad.  Rows k >= K are zero.
+__global__ void __launch_bounds__(256) pack_regrouped_kernel(const float *__restrict__ w, int K, int C, int R, int S, int sf, int Re,
+                                                             int Se, int er, int es, int k_alloc, __nv_bfloat16 *__restrict__ out) {
+    const size_t total = (size_t)k_alloc * Re * Se * 16;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        const int ch = (int)(e % 16);
+        size_t t = e / 16;
+        const int se = (int)(t % Se); t /= Se;
+        const int re = (int)(t % Re);
+        const int k = (int)(t / Re);
+        float v = 0.f;
+        const int blk = ch / C, c = ch - blk * C;
+        if (k < K && blk < sf * sf) {
+            const int dy = blk / sf, dx = blk - dy * sf;
+            const int r = sf * re + dy - er, s2 = sf * se + dx - es;
+            if (r >= 0 && r < R && s2 >= 0 && s2 < S) v = w[(((size_t)k * C + c) * R + r) * S + s2];
+        }
+        out[e] = __float2bfloat16_rn(v);
+    }
+}
+
+cprune_status pack_conv_patch(const cprune_plan *plan, const float *w, void *w_packed, cudaStream_t st) {
+    const cprune_plan_info &i = plan->info;
+    PatchGeometry g;
+    if (!patch_geometry(i, &g) || !g.stem) return CPRUNE_ERR_INTERNAL;
+    const size_t total = (size_t)i.k_alloc * g.Re * g.Se * 16;
+    size_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    pack_regrouped_kernel<<<(unsigned)blocks, 256, 0, st>>>(w, i.K, i.C, i.R, i.S, g.sf, g.Re, g.Se, g.sf * g.pad_lo - i.pad,
+                                                           g.sf * g.pad_lo - i.pad, i.k_alloc, (__nv_bfloat16 *)w_packed);
+    CPRUNE_LAUNCH_CHECK("pack_regrouped_kernel");
+    return CPRUNE_OK;
+}
+
+size_t packed_weight_bytes_patch(const cprune_plan *plan) {
+    const cprune_plan_info &i = plan->info;
+    PatchGeometry g;
+    if (!patch_geometry(i, &g) || !g.stem) return 0;
+    return (size_t)i.k_alloc * g.Re * g.Se * 32;
+}
+
 cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res, void *y,
-                                cudaStream_t st) {
+                                void *scratch, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
     const PatchTiling &t = plan->pt;
-    const int Wp = i.W + 2 * i.pad;
+    PatchGeometry g;
+    if (!patch_geometry(i, &g)) return CPRUNE_ERR_INTERNAL;
+    const int Wp = g.Wp;
+    const void *xe = x;        // the tensor the patch loads read
+    if (g.stem) {
+        if (!scratch) return CPRUNE_ERR_INVALID_ARG;
+        const long long total = (long long)i.N * g.He * g.WP;
+        long long blocks = (total + 255) / 256;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        regroup_kernel<<<(unsigned)blocks, 256, 0, st>>>((const bf16x8 *)x, i.N, i.H, i.W, i.C, g.sf, g.pad_lo, g.WP, (uint4 *)scratch);
+        CPRUNE_LAUNCH_CHECK("regroup_kernel");
+        xe = scratch;
+    }
     CUtensorMap tm_x, tm_w, tm_y, tm_res;
     {
         std::lock_guard<std::mutex> lock(plan->mu);
-        if (plan->map_x != x) {
-            const unsigned long long dims[4] = {(unsigned long long)i.c_pad, (unsigned long long)i.W, (unsigned long long)i.H,
-                                                (unsigned long long)i.N};
-            const unsigned long long strides[3] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.W * i.c_pad * 2,
-                                                   (unsigned long long)i.H * i.W * i.c_pad * 2};
-            const unsigned box[4] = {64, (unsigned)Wp, (unsigned)(t.TH + i.R - 1), 1};
-            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_a, x, 4, dims, strides, box);
-            if (s != CPRUNE_OK) return s;
-            plan->map_x = x;
+        if (plan->map_x != xe) {
+            if (g.stem) {
+                // rows of 64 values = four consecutive regrouped pixels; start positions are one pixel (32 bytes) apart
+                const unsigned long long dims[4] = {64, (unsigned long long)i.Q, (unsigned long long)g.He, (unsigned long long)i.N};
+                const unsigned long long strides[3] = {32, (unsigned long long)g.WP * 32, (unsigned long long)g.He * g.WP * 32};
+                const unsigned box[4] = {64, (unsigned)Wp, (unsigned)(t.TH + g.kR - 1), 1};
+                cprune_status s = encode_tiled_bf16_swz(&plan->tm_a, xe, 4, dims, strides, box, 128, true);
+                if (s != CPRUNE_OK) return s;
+            } else {
+                const unsigned long long dims[4] = {(unsigned long long)i.c_pad, (unsigned long long)i.W, (unsigned long long)i.H,
+                                                    (unsigned long long)i.N};
+                const unsigned long long strides[3] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.W * i.c_pad * 2,
+                                                       (unsigned long long)i.H * i.W * i.c_pad * 2};
+                const unsigned box[4] = {64, (unsigned)Wp, (unsigned)(t.TH + g.kR - 1), 1};
+                cprune_status s = encode_tiled_bf16_swz(&plan->tm_a, xe, 4, dims, strides, box, 128, true);
+                if (s != CPRUNE_OK) return s;
+            }
+            plan->map_x = xe;
         }
         if (plan->map_w != w) {
-            const unsigned long long dims[3] = {(unsigned long long)i.c_pad, (unsigned long long)(i.R * i.S), (unsigned long long)i.k_alloc};
-            const unsigned long long strides[2] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.R * i.S * i.c_pad * 2};
+            // filters [k_alloc][taps][channels of a tap]; a stem's tap is a filter row: Se pixels of 16 channels
+            const unsigned long long ctap = g.stem ? (unsigned long long)g.Se * 16 : (unsigned long long)i.c_pad;
+            const unsigned long long taps = (unsigned long long)(g.kR * g.kS);
+            const unsigned long long dims[3] = {ctap, taps, (unsigned long long)i.k_alloc};
+            const unsigned long long strides[2] = {ctap * 2, taps * ctap * 2};
             const unsigned box[3] = {64, 1, (unsigned)t.FT};
-            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_b, w, 3, dims, strides, box);
+            cprune_status s = encode_tiled_bf16_swz(&plan->tm_b, w, 3, dims, strides, box, 128, true);
             if (s != CPRUNE_OK) return s;
             plan->map_w = w;
         }
@@ -582,22 +718,22 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
             const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)i.out_w * i.k_pad * 2,
                                                    (unsigned long long)i.out_h * i.out_w * i.k_pad * 2};
             const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
-            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_y, y, 4, dims, strides, box, false);
+            cprune_status s = encode_tiled_bf16_swz(&plan->tm_y, y, 4, dims, strides, box, 128, false);
             if (s != CPRUNE_OK) return s;
             plan->map_y = y;
         }
-        std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
-        std::memcpy(&tm_w, &plan->tm_b, sizeof(CUtensorMap));
         if (res && plan->map_res != res) {
             const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)i.Q, (unsigned long long)i.P,
                                                 (unsigned long long)i.N};
             const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)i.Q * i.k_pad * 2,
                                                    (unsigned long long)i.P * i.Q * i.k_pad * 2};
             const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
-            cprune_status s = encode_tiled_bf16_sw128(&plan->tm_res, res, 4, dims, strides, box);
+            cprune_status s = encode_tiled_bf16_swz(&plan->tm_res, res, 4, dims, strides, box, 128, true);
             if (s != CPRUNE_OK) return s;
             plan->map_res = res;
         }
+        std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
+        std::memcpy(&tm_w, &plan->tm_b, sizeof(CUtensorMap));
         std::memcpy(&tm_y, &plan->tm_y, sizeof(CUtensorMap));
         std::memcpy(&tm_res, res ? &plan->tm_res : &plan->tm_y, sizeof(CUtensorMap));
     }
@@ -612,15 +748,17 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     }
     PatchParams p;
     p.P = i.P; p.Q = i.Q; p.Wp = Wp; p.TH = t.TH; p.tiles_per_img = t.tiles_per_img;
-    p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.FT = t.FT; p.MT = t.MT; p.R = i.R; p.S = i.S; p.pad = i.pad;
-    p.cblks = (i.c_pad + 63) / 64;
-    p.ksteps_last = (i.c_pad - (p.cblks - 1) * 64 + 15) / 16;
+    p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.FT = t.FT; p.MT = t.MT; p.R = g.kR; p.S = g.kS; p.pad = g.pad_lo; p.pad_w = g.pad_w;
+    p.cblks = g.cblks;
+    p.ksteps_last = g.ksteps_last;
     p.k_pad = i.k_pad;
     p.act = plan->opts.activation;
     p.wstages = t.wstages; p.resident = t.resident; p.acc_bufs = t.acc_bufs; p.staging_bufs = t.staging_bufs;
     p.pool = plan->fused_pool;
     p.patch_bytes = t.patch_bytes;
-    p.patch_box_bytes = Wp * (t.TH + i.R - 1) * 128;
+    p.patch_box_bytes = Wp * (t.TH + g.kR - 1) * 128;
+    p.rb16 = 8;
+    p.w_stage_bytes = t.FT * 128;
     p.bias = b;
     p.res = (const __nv_bfloat16 *)res;
     p.y = (__nv_bfloat16 *)y;

@@ -749,8 +749,8 @@ cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, con
     return CPRUNE_OK;
 }
 
-cprune_status encode_tiled_bf16_sw128(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
-                                      const unsigned long long *strides_bytes, const unsigned *box, bool for_loads) {
+cprune_status encode_tiled_bf16_swz(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
+                                    const unsigned long long *strides_bytes, const unsigned *box, int swizzle_bytes, bool for_loads) {
     cprune_status st = load_driver_entry_points();
     if (st != CPRUNE_OK) return st;
     cuuint64_t d[5], s[4];
@@ -758,7 +758,7 @@ cprune_status encode_tiled_bf16_sw128(CUtensorMap *map, const void *ptr, int ran
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; e[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) s[i] = strides_bytes[i];
     CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(ptr), d, s, b, e,
-                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_32B,
                                 for_loads ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(swizzle 128)");
@@ -977,7 +977,7 @@ static int sm_count() {
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
                                  void *y, void *partial, cudaStream_t st) {
     const cprune_plan_info &i = plan->info;
-    if (plan->patch) return launch_conv_patch(plan, x, w, b, res, y, st);
+    if (plan->patch) return launch_conv_patch(plan, x, w, b, res, y, partial, st);
     CUtensorMap tm_x, tm_w, tm_y, tm_res, tm_id;
     const bool split = plan->splits > 1;
     if (split && !partial) return CPRUNE_ERR_INVALID_ARG;

@@ -98,6 +98,11 @@ cprune_status cprune_pack_weights(const cprune_plan *plan, const float *w, const
         CPRUNE_LAUNCH_CHECK("pad_bias_kernel");
         return CPRUNE_OK;
     }
+    if (i.kernel == CPRUNE_KERNEL_TENSOR && plan->patch && plan->narrow) {
+        pad_bias_kernel<<<(i.k_alloc + 255) / 256, 256, 0, st>>>(b, i.K, i.k_alloc, b_packed);
+        CPRUNE_LAUNCH_CHECK("pad_bias_kernel");
+        return pack_conv_patch(plan, w, w_packed, st);
+    }
     const int s_out = (i.kernel == CPRUNE_KERNEL_TENSOR && plan->s_packed > 0) ? plan->s_packed : i.S;
     return pack_dense(w, b, i.K, i.C, i.R, i.S, s_out, i.k_alloc, i.c_pad, w_packed, b_packed, st);
 }

@@ -71,11 +71,13 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     const double rs = (double)i.R * i.S;
     const int s_packed = (family == CPRUNE_KERNEL_TENSOR && pl->s_packed > 0) ? pl->s_packed : i.S;
     i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * s_packed * i.c_pad * 2;
+    if (family == CPRUNE_KERNEL_TENSOR && pl->patch && pl->narrow) i.packed_weight_bytes = packed_weight_bytes_patch(pl);
     i.packed_bias_bytes = (size_t)i.k_alloc * sizeof(float);
     // workspace: [unpooled conv output if a pool follows][split-K partial sums]
     const bool separate_pool = pl->opts.pool == CPRUNE_POOL_MAX2X2 && !(family == CPRUNE_KERNEL_TENSOR && pl->fused_pool);
     pl->pool_bytes = separate_pool ? ((size_t)i.N * i.P * i.Q * i.k_pad * 2 + 255) / 256 * 256 : 0;
-    i.workspace_bytes = pl->pool_bytes + (family == CPRUNE_KERNEL_TENSOR ? pl->partial_bytes : 0);
+    // (patch kernel on a regrouped stem: the regrouped input takes the place of the partial sums)
+    i.workspace_bytes = pl->pool_bytes + (family == CPRUNE_KERNEL_TENSOR ? pl->partial_bytes + pl->pre_bytes : 0);
     i.algorithmic_bytes = 2.0 * ((double)i.N * i.H * i.W * i.C + (double)i.N * i.out_h * i.out_w * i.K +
                                  (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
                                  (double)i.K * (i.C / i.groups) * rs) + 4.0 * i.K;
@@ -175,7 +177,7 @@ cprune_status cprune_task_run(cprune_plan *plan, const void *x, const void *w_pa
     const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2 && !(i.kernel == CPRUNE_KERNEL_TENSOR && plan->fused_pool);
     if (i.workspace_bytes && !workspace) return CPRUNE_ERR_INVALID_ARG;
     void *conv_out = pool ? workspace : y;
-    void *partial = plan->partial_bytes ? (void *)((char *)workspace + plan->pool_bytes) : nullptr;
+    void *partial = (plan->partial_bytes || plan->pre_bytes) ? (void *)((char *)workspace + plan->pool_bytes) : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
     cprune_status s;
     switch (i.kernel) {

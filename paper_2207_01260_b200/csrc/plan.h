@@ -41,7 +41,9 @@ struct cprune_plan {
     size_t partial_bytes = 0;       // float32 partial sums in the workspace
     int small_c = 0;                // 3-channel stems: 1 = 8 taps x 8 channels per K block, 2 = pixel pairs
     int s_packed = 0;               // filter taps per row in the packed weights (S, or S + 1 in pair mode)
-    int patch = 0;                  // 1: stride-1 task on the patch kernel (conv_patch.cu)
+    int patch = 0;                  // 1: task on the patch kernel (conv_patch.cu)
+    int narrow = 0;                 // patch kernel on a regrouped 16-channel input (stems with few channels)
+    size_t pre_bytes = 0;           // regrouped input in the workspace
     PatchTiling pt = {};
 };
 
@@ -60,10 +62,14 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
 // stride-1 R x S > 1 tasks with the input patch resident in shared memory (part of the tensor family)
 cprune_status plan_conv_patch(cprune_plan *plan);   // UNSUPPORTED if the task is not eligible or would waste the tile
 cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
-                                void *y, cudaStream_t st);
-// tiled bf16 tensor map with the 128-byte swizzle (inner box extent 64 elements), out-of-bounds elements read as zero
-cprune_status encode_tiled_bf16_sw128(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
-                                      const unsigned long long *strides_bytes, const unsigned *box, bool for_loads = true);
+                                void *y, void *scratch, cudaStream_t st);
+// filters of a regrouped stem (plan->narrow) and their size
+cprune_status pack_conv_patch(const cprune_plan *plan, const float *w, void *w_packed, cudaStream_t st);
+size_t packed_weight_bytes_patch(const cprune_plan *plan);
+// tiled bf16 tensor map with a 128- or 32-byte swizzle (inner box extent 64 or 16 elements); out-of-bounds
+// elements read as zero
+cprune_status encode_tiled_bf16_swz(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
+                                    const unsigned long long *strides_bytes, const unsigned *box, int swizzle_bytes, bool for_loads);
 // tiled bf16 tensor map without swizzle, out-of-bounds elements read as zero
 cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
                                 const unsigned long long *strides_bytes, const unsigned *box);

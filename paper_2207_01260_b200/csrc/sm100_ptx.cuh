@@ -166,9 +166,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 
 // The same descriptor split into words: the high word is a constant, the low word holds the start address
 // (16-byte units) and the unused leading-offset field, so that address arithmetic is a 32-bit add.
+// High word for 128-byte rows (128-byte swizzle, 8-row groups 1024 bytes apart) and for 32-byte rows (32-byte
+// swizzle, 8-row groups 256 bytes apart).
 constexpr uint32_t DESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo_sw128(uint32_t addr) { return ((addr >> 4) & 0x3FFFu) | (1u << 16); }
-__device__ __forceinline__ void umma_bf16_sw128(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+constexpr uint32_t DESC_HI_SW32 = (256u >> 4) | (1u << 14) | (6u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr) { return ((addr >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ void umma_bf16_words(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                                uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
         "mov.b64 da, {%1, %4};\n\t"
@@ -176,7 +180,7 @@ __device__ __forceinline__ void umma_bf16_sw128(uint32_t d_tmem, uint32_t a_lo, 
         "setp.ne.b32 p, %5, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
         :
-        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI_SW128), "r"(accumulate)
+        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(desc_hi), "r"(accumulate)
         : "memory");
 }
 
