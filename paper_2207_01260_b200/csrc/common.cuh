@@ -30,6 +30,35 @@ cprune_status cuda_fail(cudaError_t e, const char *what);
         if (e__ != cudaSuccess) return ::cprune::cuda_fail(e__, name); \
     } while (0)
 
+// Programmatic dependent launch.  A kernel of a model's launch chain lets its successor start as early as possible
+// (pdl_trigger) and waits for its predecessor's results (pdl_wait) only after its own set-up, so that launch
+// latency and set-up overlap the predecessor's tail.  Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// True while the calling thread enqueues a chain whose kernels may overlap their predecessors' tails.
+bool chain_launch_enabled();
+void set_chain_launch(bool on);
+
+// Launches a kernel that calls pdl_wait() before it touches global memory; inside a chain the launch carries the
+// programmatic-serialization attribute.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (chain_launch_enabled()) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
 

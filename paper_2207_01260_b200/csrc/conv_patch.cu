@@ -99,6 +99,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1)
 conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res, const PatchParams p) {
     extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - raw);
@@ -158,6 +159,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // set-up done: from here on the kernel reads what its predecessor wrote
+    pdl_wait();
     const uint32_t tmem_base = *tmem_slot;
     const int total_items = p.tiles_m * p.tiles_n;
 
@@ -594,6 +597,8 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
 // out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
 __global__ void __launch_bounds__(256) regroup_kernel(const bf16x8 *__restrict__ x, int N, int H, int W, int C, int sf, int pad_lo,
                                                       int WP, uint4 *__restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
     const int H2 = H / sf, W2 = W / sf;
     const long long total = (long long)N * H2 * WP;
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
@@ -673,8 +678,8 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
         const long long total = (long long)i.N * g.He * g.WP;
         long long blocks = (total + 255) / 256;
         if (blocks > 148 * 16) blocks = 148 * 16;
-        regroup_kernel<<<(unsigned)blocks, 256, 0, st>>>((const bf16x8 *)x, i.N, i.H, i.W, i.C, g.sf, g.pad_lo, g.WP, (uint4 *)scratch);
-        CPRUNE_LAUNCH_CHECK("regroup_kernel");
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel, dim3((unsigned)blocks), dim3(256), 0, st, (const bf16x8 *)x, i.N, i.H, i.W, i.C, g.sf, g.pad_lo,
+                                         g.WP, (uint4 *)scratch));
         xe = scratch;
     }
     CUtensorMap tm_x, tm_w, tm_y, tm_res;
@@ -770,8 +775,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
     const int grid = total < sms ? total : sms;
-    conv_patch_kernel<<<grid, PK_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, p);
-    CPRUNE_LAUNCH_CHECK("conv_patch_kernel");
+    CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     return CPRUNE_OK;
 }
 

@@ -97,6 +97,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
                const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res,
                const __grid_constant__ CUtensorMap tm_id, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     uint8_t *smem = smem_raw + (base - raw);
@@ -143,6 +144,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                                            // set-up done: from here on the predecessor's results are read
     const uint32_t tmem_base = *tmem_slot;
 
     const int k_alloc = p.tiles_n * p.FT;     // row length of the float32 partial sums (split-K)
@@ -670,6 +672,8 @@ __global__ void __launch_bounds__(256) splitk_finalize_kernel(const float *__res
                                                               int k_alloc, int k8, const float *__restrict__ bias,
                                                               const bf16x8 *__restrict__ res, int act, int pool_q,
                                                               bf16x8 *__restrict__ y) {
+    pdl_trigger();
+    pdl_wait();
     const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long out_pixels = pool_q ? M / 4 : M;
     if (e >= out_pixels * k8) return;
@@ -1034,20 +1038,18 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     const int grid = total < sm_count() ? total : sm_count();
     const bool pool_in_kernel = plan->fused_pool && !split;
     if (plan->orient == ORIENT_PIX) {
-        if (pool_in_kernel) conv_tc_kernel<ORIENT_PIX, 1><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
-        else conv_tc_kernel<ORIENT_PIX, 0><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+        if (pool_in_kernel) CPRUNE_CUDA_CHECK(launch_chained(conv_tc_kernel<ORIENT_PIX, 1>, dim3(grid), dim3(TC_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, tm_id, p));
+        else CPRUNE_CUDA_CHECK(launch_chained(conv_tc_kernel<ORIENT_PIX, 0>, dim3(grid), dim3(TC_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, tm_id, p));
     } else {
-        if (pool_in_kernel) conv_tc_kernel<ORIENT_FILT, 1><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
-        else conv_tc_kernel<ORIENT_FILT, 0><<<grid, TC_THREADS, plan->smem_bytes, st>>>(tm_x, tm_w, tm_y, tm_res, tm_id, p);
+        if (pool_in_kernel) CPRUNE_CUDA_CHECK(launch_chained(conv_tc_kernel<ORIENT_FILT, 1>, dim3(grid), dim3(TC_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, tm_id, p));
+        else CPRUNE_CUDA_CHECK(launch_chained(conv_tc_kernel<ORIENT_FILT, 0>, dim3(grid), dim3(TC_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, tm_id, p));
     }
     CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
     if (split) {
         const long long elems = (plan->fused_pool ? p.M / 4 : p.M) * (i.k_pad / 8);
-        splitk_finalize_kernel<<<(unsigned)ceil_div(elems, 256), 256, 0, st>>>((const float *)partial, plan->splits, p.M,
-                                                                              i.k_alloc, i.k_pad / 8, b, (const bf16x8 *)res,
-                                                                              plan->opts.activation,
-                                                                              plan->fused_pool ? i.Q : 0, (bf16x8 *)y);
-        CPRUNE_LAUNCH_CHECK("splitk_finalize_kernel");
+        CPRUNE_CUDA_CHECK(launch_chained(splitk_finalize_kernel, dim3((unsigned)ceil_div(elems, 256)), dim3(256), 0, st, (const float *)partial,
+                                         plan->splits, p.M, i.k_alloc, i.k_pad / 8, b, (const bf16x8 *)res, plan->opts.activation,
+                                         plan->fused_pool ? i.Q : 0, (bf16x8 *)y));
     }
     return CPRUNE_OK;
 }

@@ -37,6 +37,8 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
     __shared__ __align__(8) unsigned long long bar;
     __shared__ int failed;
 
+    pdl_trigger();
+    pdl_wait();
     int bid = blockIdx.x;
     const int cb = bid % p.cblocks; bid /= p.cblocks;
     const int tw = bid % p.tiles_w; bid /= p.tiles_w;
@@ -238,8 +240,8 @@ cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, 
     }
     if (smem > 100 * 1024) return CPRUNE_ERR_UNSUPPORTED;
     const int threads = ((p.TW * p.G + 31) / 32) * 32;
-    if (i.stride == 1) depthwise3x3_kernel<1><<<(unsigned)blocks, threads, smem, st>>>(tm, p);
-    else depthwise3x3_kernel<2><<<(unsigned)blocks, threads, smem, st>>>(tm, p);
+    if (i.stride == 1) CPRUNE_CUDA_CHECK(launch_chained(depthwise3x3_kernel<1>, dim3((unsigned)blocks), dim3(threads), (size_t)smem, st, tm, p));
+    else CPRUNE_CUDA_CHECK(launch_chained(depthwise3x3_kernel<2>, dim3((unsigned)blocks), dim3(threads), (size_t)smem, st, tm, p));
     CPRUNE_LAUNCH_CHECK("depthwise3x3_kernel");
     return CPRUNE_OK;
 }

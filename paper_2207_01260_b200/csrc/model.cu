@@ -49,7 +49,17 @@ static void *tensor_ptr(const cprune_model *m, int id) {
     return it == m->tensors.end() ? nullptr : (void *)(m->arena + it->second.offset);
 }
 
+static cprune_status enqueue_chain(cprune_model *m, const float *x, float *logits, cudaStream_t st);
+
+// The kernels of one pass are launched as a chain: each may start while its predecessor drains (see common.cuh).
 static cprune_status enqueue(cprune_model *m, const float *x, float *logits, cudaStream_t st) {
+    set_chain_launch(true);
+    cprune_status s = enqueue_chain(m, x, logits, st);
+    set_chain_launch(false);
+    return s;
+}
+
+static cprune_status enqueue_chain(cprune_model *m, const float *x, float *logits, cudaStream_t st) {
     cprune_status s = cprune_cast_input(x, (size_t)m->N * m->H * m->W, m->C, tensor_ptr(m, 0), st);
     if (s != CPRUNE_OK) return s;
     for (size_t t = 0; t < m->tasks.size(); ++t) {

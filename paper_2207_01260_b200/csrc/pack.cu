@@ -41,6 +41,8 @@ __global__ void pad_bias_kernel(const float *__restrict__ b, int K, int k_alloc,
 
 // one thread per (pixel, group of 8 output lanes)
 __global__ void cast_input_kernel(const float *__restrict__ x, size_t pixels, int C, int c_pad, bf16x8 *__restrict__ y) {
+    pdl_trigger();
+    pdl_wait();
     int groups = c_pad / 8;
     size_t total = pixels * groups;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
@@ -118,9 +120,8 @@ cprune_status cprune_cast_input(const float *x, size_t pixels, int C, void *y, v
     if (!x || !y || C <= 0) return CPRUNE_ERR_INVALID_ARG;
     if (pixels == 0) return CPRUNE_OK;
     int c_pad = cprune_padded_channels(C);
-    cast_input_kernel<<<grid_for(pixels * (c_pad / 8), 256), 256, 0, (cudaStream_t)stream>>>(x, pixels, C, c_pad,
-                                                                                            (bf16x8 *)y);
-    CPRUNE_LAUNCH_CHECK("cast_input_kernel");
+    CPRUNE_CUDA_CHECK(launch_chained(cast_input_kernel, dim3(grid_for(pixels * (c_pad / 8), 256)), dim3(256), 0, (cudaStream_t)stream, x, pixels, C,
+                                     c_pad, (bf16x8 *)y));
     return CPRUNE_OK;
 }
 

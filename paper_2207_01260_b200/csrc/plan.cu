@@ -2,6 +2,7 @@
 // properties map to one task, and each task keeps one program).  A plan is a pure function of its
 // key (shape + fused-epilogue options); planning launches nothing and needs no device.
 #include <array>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 
@@ -9,6 +10,13 @@
 #include "plan.h"
 
 namespace cprune {
+
+static thread_local bool g_chain_launch = false;
+bool chain_launch_enabled() { return g_chain_launch; }
+void set_chain_launch(bool on) {
+    const char *off = getenv("CPRUNE_NO_PDL");     // measurement override
+    g_chain_launch = on && !(off && off[0] == '1');
+}
 
 using PlanKey = std::array<int, 14>;
 

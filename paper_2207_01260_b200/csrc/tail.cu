@@ -8,6 +8,8 @@ namespace cprune {
 __global__ void __launch_bounds__(256) maxpool_kernel(const bf16x8 *__restrict__ x, int N, int H, int W, int c8,
                                                       int P, int Q, int k, int stride, int pad,
                                                       bf16x8 *__restrict__ y) {
+    pdl_trigger();
+    pdl_wait();
     long long total = (long long)N * P * Q * c8;
     long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= total) return;
@@ -35,26 +37,44 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const bf16x8 *__restrict__
     y[e] = pack8(m);
 }
 
-// one thread per (n, channel group): mean over H*W in float32, stored as bf16
-__global__ void __launch_bounds__(128) gap_kernel(const bf16x8 *__restrict__ x, int N, int HW, int c8,
+// One block per (image, 32 channel groups): 8 pixel lanes x 32 channel groups; each thread sums every 8th pixel of
+// its channel group in float32, the lanes are added through shared memory in a fixed order, mean stored as bf16.
+__global__ void __launch_bounds__(256) gap_kernel(const bf16x8 *__restrict__ x, int N, int HW, int c8,
                                                   bf16x8 *__restrict__ y) {
-    int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= N * c8) return;
-    int cg = e % c8, n = e / c8;
+    __shared__ float part[8][32][9];
+    pdl_trigger();
+    pdl_wait();
+    const int blocks_per_img = (c8 + 31) / 32;
+    const int n = blockIdx.x / blocks_per_img;
+    const int cg = (blockIdx.x - n * blocks_per_img) * 32 + (threadIdx.x & 31);
+    const int pl = threadIdx.x >> 5;
     float s[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) s[i] = 0.f;
-    const bf16x8 *px = x + (size_t)n * HW * c8 + cg;
-    for (int i = 0; i < HW; ++i) {
-        float f[8];
-        unpack8(ldg8(px + (size_t)i * c8), f);
+    if (cg < c8) {
+        const bf16x8 *px = x + (size_t)n * HW * c8 + cg;
+        for (int i = pl; i < HW; i += 8) {
+            float f[8];
+            unpack8(ldg8(px + (size_t)i * c8), f);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s[j] += f[j];
+            for (int j = 0; j < 8; ++j) s[j] += f[j];
+        }
     }
-    float inv = 1.f / (float)HW;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) s[j] *= inv;
-    y[e] = pack8(s);
+    for (int j = 0; j < 8; ++j) part[pl][threadIdx.x & 31][j] = s[j];
+    __syncthreads();
+    if (pl == 0 && cg < c8) {
+        float t[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) t[j] = 0.f;
+        for (int l = 0; l < 8; ++l)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) t[j] += part[l][threadIdx.x & 31][j];
+        const float inv = 1.f / (float)HW;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) t[j] *= inv;
+        y[(size_t)n * c8 + cg] = pack8(t);
+    }
 }
 
 // one warp per (output feature o, group of NB images): the warp reads the weight row once and
@@ -64,6 +84,8 @@ template <int NB>
 __global__ void __launch_bounds__(256) fc_kernel(const bf16x8 *__restrict__ x, int N, int in8,
                                                  const bf16x8 *__restrict__ w, const float *__restrict__ b, int out,
                                                  int out_pad, int act, int out_is_f32, void *__restrict__ y) {
+    pdl_trigger();
+    pdl_wait();
     const int ngroups = (N + NB - 1) / NB;
     const long long widx = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -109,9 +131,8 @@ cprune_status launch_maxpool(const void *x, int N, int H, int W, int c_pad, int 
     if (total == 0) return CPRUNE_OK;
     long long blocks = ceil_div(total, 256);
     if (blocks > 0x7fffffffLL) return CPRUNE_ERR_UNSUPPORTED;
-    maxpool_kernel<<<(unsigned)blocks, 256, 0, st>>>((const bf16x8 *)x, N, H, W, c_pad / 8, P, Q, k, stride, pad,
-                                                     (bf16x8 *)y);
-    CPRUNE_LAUNCH_CHECK("maxpool_kernel");
+    CPRUNE_CUDA_CHECK(launch_chained(maxpool_kernel, dim3((unsigned)blocks), dim3(256), 0, st, (const bf16x8 *)x, N, H, W, c_pad / 8, P, Q, k,
+                                     stride, pad, (bf16x8 *)y));
     return CPRUNE_OK;
 }
 
@@ -132,8 +153,8 @@ cprune_status cprune_maxpool(const void *x, int N, int H, int W, int C, int k, i
 cprune_status cprune_global_avgpool(const void *x, int N, int H, int W, int C, void *y, void *stream) {
     if (!x || !y || N <= 0 || H <= 0 || W <= 0 || C <= 0) return CPRUNE_ERR_INVALID_ARG;
     int c8 = cprune_padded_channels(C) / 8;
-    gap_kernel<<<(N * c8 + 127) / 128, 128, 0, (cudaStream_t)stream>>>((const bf16x8 *)x, N, H * W, c8, (bf16x8 *)y);
-    CPRUNE_LAUNCH_CHECK("gap_kernel");
+    CPRUNE_CUDA_CHECK(launch_chained(gap_kernel, dim3(N * ((c8 + 31) / 32)), dim3(256), 0, (cudaStream_t)stream, (const bf16x8 *)x, N, H * W, c8,
+                                     (bf16x8 *)y));
     return CPRUNE_OK;
 }
 
@@ -143,9 +164,8 @@ cprune_status cprune_fc(const void *x, int N, int in, const void *w_packed, cons
     int in8 = cprune_padded_channels(in) / 8, out_pad = cprune_padded_channels(out);
     const int warps = 8;
     const long long total_warps = (long long)out_pad * ((N + 7) / 8);
-    fc_kernel<8><<<(unsigned)((total_warps + warps - 1) / warps), warps * 32, 0, (cudaStream_t)stream>>>(
-        (const bf16x8 *)x, N, in8, (const bf16x8 *)w_packed, b_packed, out, out_pad, act, out_is_f32, y);
-    CPRUNE_LAUNCH_CHECK("fc_kernel");
+    CPRUNE_CUDA_CHECK(launch_chained(fc_kernel<8>, dim3((unsigned)((total_warps + warps - 1) / warps)), dim3(warps * 32), 0, (cudaStream_t)stream,
+                                     (const bf16x8 *)x, N, in8, (const bf16x8 *)w_packed, b_packed, out, out_pad, act, out_is_f32, y));
     return CPRUNE_OK;
 }
 
