@@ -39,11 +39,18 @@ def test_status_strings_and_padding(cp):
 def test_plan_shapes_and_families(cp):
     p = cp.cprune_task_plan(64, 64, 56, 56, 44, 3, 3, 1, 1)
     assert (p.P, p.Q, p.c_pad, p.k_pad) == (56, 56, 64, 48)
-    # K <= 128: filters sit on the 128-row side of the MMA and a tile covers 256 pixels
-    assert cp.KERNEL_NAMES[p.kernel] == "tensor" and p.tile_m == 256 and p.tile_n == 128
-    assert p.tiles_m == 64 * 56 * 56 // 256 and p.tiles_n == 1 and p.k_alloc == 128
+    # stride-1 3x3 with many tiles: patch kernel, a tile is 4 whole output rows (2 x 128 accumulator rows, 58 per
+    # image row with the two wrap-around columns), all 48 padded filters in one MMA
+    assert cp.KERNEL_NAMES[p.kernel] == "tensor" and p.tile_m == 256 and p.tile_n == 48
+    assert p.tiles_m == 64 * 14 and p.tiles_n == 1 and p.k_alloc == 48 and p.workspace_bytes == 0
     q = cp.cprune_task_plan(64, 256, 14, 14, 358, 3, 3, 1, 1)
-    assert q.tile_m == 128 and q.tile_n % 16 == 0 and q.tiles_n * q.tile_n >= 358 and q.k_alloc == q.tiles_n * q.tile_n
+    assert q.tile_m in (128, 256) and q.tile_n % 16 == 0 and q.tiles_n * q.tile_n >= 358 and q.k_alloc == q.tiles_n * q.tile_n
+    # 1x1 and stride-2 tasks stay on the im2col kernel: K <= 128 puts the filters on the 128-row side, 256 pixels a tile
+    r = cp.cprune_task_plan(64, 64, 56, 56, 128, 1, 1, 2, 0)
+    assert cp.KERNEL_NAMES[r.kernel] == "tensor" and r.tile_m == 256 and r.tile_n == 128 and r.k_alloc == 128
+    # a stem with enough tiles runs on the patch kernel and asks for room for the regrouped input
+    s = cp.cprune_task_plan(64, 3, 224, 224, 64, 7, 7, 2, 3)
+    assert cp.KERNEL_NAMES[s.kernel] == "tensor" and s.workspace_bytes >= 64 * 112 * 115 * 32
     assert p.flops == 2.0 * 64 * 44 * 64 * 56 * 56 * 9
     assert p.padded_flops >= p.flops
     p = cp.cprune_task_plan(1, 3, 224, 224, 64, 7, 7, 2, 3)
