@@ -30,7 +30,7 @@ import numpy as np  # noqa: E402
 
 # DRAM bytes (read + write) of all conv_tc_kernel launches of one model pass, from the ncu capture summarised in
 # profiles/conv_tc_resnet18_b64_dram_traffic.md; None where no capture of the current kernel exists.
-CONV_TC_DRAM_BYTES_PER_STEP = {"resnet18": 415.9e6, "mobilenet_v2": None, "vgg16_cifar": None}
+DRAM_BYTES_PER_STEP = {}
 
 WORKLOADS = {"resnet18": ("resnet18", 64), "mobilenet_v2": ("mobilenet_v2", 64), "vgg16_cifar": ("vgg16_cifar", 128)}
 
@@ -251,7 +251,12 @@ def main():
     if rank == 0 and not args.no_task_times:
         peaks = measured_peaks()
         per_task = net_task_times(cp, net, table, x, reps=5)
-        tens = [t for t in per_task if t["kernel"] == "tensor"]
+        # the tensor family has two kernels; the roofline object describes the one that takes more of the step
+        tens_all = [t for t in per_task if t["kernel"] == "tensor"]
+        by_variant = {v: [t for t in tens_all if t["variant"] == v] for v in (0, 1)}
+        top = max((0, 1), key=lambda v: sum(t["ms"] for t in by_variant[v]))
+        tens = by_variant[top]
+        tens_name = "conv_patch_kernel" if top == 1 else "conv_tc_kernel"
         dw = [t for t in per_task if t["kernel"] == "depthwise"]
         t_tens, t_dw = sum(t["ms"] for t in tens), sum(t["ms"] for t in dw)
         if t_dw > t_tens and dw:
@@ -263,9 +268,9 @@ def main():
         elif tens:
             tf = sum(t["flops"] for t in tens) / 1e12
             ach = tf / (t_tens * 1e-3)
-            roof = {"kernel": "conv_tc_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+            roof = {"kernel": tens_name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
-                    "traffic": CONV_TC_DRAM_BYTES_PER_STEP.get(args.workload),
+                    "traffic": DRAM_BYTES_PER_STEP.get((args.workload, tens_name)),
                     "traffic_note": "DRAM bytes of all launches of this kernel in one step (ncu); algorithmic bytes alongside",
                     "algorithmic_bytes": sum(t["bytes"] for t in tens),
                     "peak_source": peaks["source"] + " (sustained bf16 GEMM)", "launches_per_step": len(tens),
@@ -453,6 +458,8 @@ def net_task_times(cp, net, table, x, reps=5):
         bufs["x"] = acts["x"]
         for l in table["layers"]:
             kind = l["kind"]
+            if l["name"] in net.absorbed:          # a max-pool that runs inside the preceding conv task
+                continue
             a = acts[l["in"]]
             if kind == "conv":
                 plan = net.plans[l["name"]]
@@ -470,7 +477,7 @@ def net_task_times(cp, net, table, x, reps=5):
                 if rep > 0:
                     times.setdefault(l["name"], []).append((s, e))
                 infos[l["name"]] = plan.info
-                acts[l["out"]] = y
+                acts[net.fused_pools[l["name"]]["out"] if l["name"] in net.fused_pools else l["out"]] = y
             elif kind == "maxpool":
                 acts[l["out"]] = cp.cprune_maxpool(a, a.shape[-1], l["k"], l["stride"], l["pad"])
             elif kind == "gap":
@@ -486,7 +493,7 @@ def net_task_times(cp, net, table, x, reps=5):
         i = infos[name]
         out.append({"name": name, "kernel": cp.KERNEL_NAMES[i["kernel"]], "C": i["C"], "K": i["K"],
                     "HW": [i["H"], i["W"]], "R": i["R"], "stride": i["stride"], "ms": ms, "flops": i["flops"],
-                    "bytes": i["algorithmic_bytes"], "tflops": i["flops"] / ms / 1e9,
+                    "variant": i["variant"], "bytes": i["algorithmic_bytes"], "tflops": i["flops"] / ms / 1e9,
                     "gbs": i["algorithmic_bytes"] / ms / 1e6, "tile_n": i["tile_n"], "tiles": i["tiles_m"] * i["tiles_n"]})
     return out
 

@@ -42,7 +42,9 @@ typedef enum {
 } cprune_status;
 
 enum { CPRUNE_ACT_NONE = 0, CPRUNE_ACT_RELU = 1, CPRUNE_ACT_RELU6 = 2 };
-enum { CPRUNE_POOL_NONE = 0, CPRUNE_POOL_MAX2X2 = 1 };
+/* max-pool applied to the activated conv result: 2x2 stride 2 (VGG blocks), or 3x3 stride 2 pad 1 (ResNet stem;
+ * padding never wins the maximum) */
+enum { CPRUNE_POOL_NONE = 0, CPRUNE_POOL_MAX2X2 = 1, CPRUNE_POOL_MAX3X3S2 = 2 };
 /* kernel families a plan can choose */
 enum { CPRUNE_KERNEL_AUTO = 0, CPRUNE_KERNEL_DIRECT = 1, CPRUNE_KERNEL_TENSOR = 2, CPRUNE_KERNEL_DEPTHWISE = 3 };
 
@@ -122,7 +124,7 @@ cprune_status cprune_gather_columns(const float *in, int outer, int cols, size_t
 typedef struct {
     int activation;   /* CPRUNE_ACT_* */
     int residual;     /* 1: a residual tensor [N][P][Q][k_pad] is added before the activation */
-    int pool;         /* CPRUNE_POOL_*: 2x2 stride-2 max-pool applied to the activated result */
+    int pool;         /* CPRUNE_POOL_*: max-pool applied to the activated result */
     int kernel;       /* CPRUNE_KERNEL_AUTO or a forced family (for tests and measurements) */
 } cprune_task_opts;
 
@@ -139,6 +141,8 @@ typedef struct {
     double flops;             /* 2 N K C P Q R S / groups */
     double algorithmic_bytes; /* bf16 x + bf16 y (+ bf16 residual) + bf16 w + fp32 b, each once */
     double padded_flops;      /* flops the chosen kernel issues, including channel and tile padding */
+    int variant;              /* tensor family: 0 = operands gathered per filter tap (im2col loads), 1 = the input patch
+                                 of a tile stays in shared memory and every tap reads it (stride-1 tasks, stems) */
 } cprune_plan_info;
 
 /* Host only; launches nothing.  opts == NULL means bias + ReLU, no residual, no pool, AUTO.

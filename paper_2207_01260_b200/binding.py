@@ -15,7 +15,7 @@ OK = 0
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA", 5: "TIMEOUT",
                 6: "INTERNAL", 7: "BAD_DATA"}
 ACT = {"none": 0, "relu": 1, "relu6": 2}
-POOL = {None: 0, "none": 0, "max2x2": 1}
+POOL = {None: 0, "none": 0, "max2x2": 1, "max3x3s2": 2}
 KERNEL = {"auto": 0, "direct": 1, "tensor": 2, "depthwise": 3}
 KERNEL_NAMES = {v: k for k, v in KERNEL.items()}
 OP_CONV, OP_MAXPOOL, OP_GAP, OP_FC = 1, 2, 3, 4
@@ -46,7 +46,7 @@ class PlanInfo(ctypes.Structure):
                                       "out_w", "c_pad", "k_pad", "kernel", "tile_m", "tile_n", "tile_k", "stages",
                                       "tiles_m", "tiles_n", "k_alloc")] + \
                [("packed_weight_bytes", c_size_t), ("packed_bias_bytes", c_size_t), ("workspace_bytes", c_size_t),
-                ("flops", c_double), ("algorithmic_bytes", c_double), ("padded_flops", c_double)]
+                ("flops", c_double), ("algorithmic_bytes", c_double), ("padded_flops", c_double), ("variant", c_int)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

@@ -50,6 +50,8 @@ constexpr int PK_BLOCK_BYTES = 16384;    // staged block: 128 slots x 64 filters
 
 struct PatchParams {
     int P, Q, Wp, TH, tiles_per_img, tiles_m, tiles_n;
+    int TW, tiles_w, step_h, step_w, org;   // tile (ty, tx) starts at output (ty * step_h + org, tx * step_w + org) and spans TH x TW
+    int out_h, out_w;                       // stored extent (after a fused pool)
     int FT, MT, R, S, pad, pad_w, cblks, ksteps_last, k_pad;   // pad: rows above the image in a patch; pad_w: columns left of it
     int act, wstages, resident, acc_bufs, staging_bufs, pool;
     int patch_bytes;       // shared memory of one patch stage
@@ -93,6 +95,17 @@ __device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint32_t a_lo, uint32
         if (commit_p) umma_commit(commit_p);
     }
     __syncwarp();
+}
+
+// First output pixel (may be -1 with the 3x3 pool, whose windows reach one pixel outside the tile's own pooled
+// pixels) and image of tile tm.
+__device__ __forceinline__ void tile_origin(const PatchParams &p, int tm, int &n, int &p0, int &q0) {
+    n = tm / p.tiles_per_img;
+    const int r = tm - n * p.tiles_per_img;
+    int ty = r, tx = 0;
+    if (p.tiles_w > 1) { ty = r / p.tiles_w; tx = r - ty * p.tiles_w; }
+    p0 = ty * p.step_h + p.org;
+    q0 = tx * p.step_w + p.org;
 }
 
 __global__ void __launch_bounds__(PK_THREADS, 1)
@@ -142,10 +155,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     // slot table: which accumulator rows hold real output pixels and where they go
     for (int e = threadIdx.x; e < 256; e += PK_THREADS) {
         int2 v = make_int2(-1, 0);
-        if (!p.pool) {
-            const int i = e / p.Wp, j = e - i * p.Wp;
-            if (e < 128 * p.MT && j < p.Q && i < p.TH) v = make_int2(e | (i << 16), (i * p.Q + j) * p.k_pad);
-        } else {
+        if (p.pool == 1) {
             const int hq = p.Q >> 1;
             const int i2 = e / hq, j2 = e - i2 * hq;
             if (i2 < (p.TH >> 1)) v = make_int2((2 * i2 * p.Wp + 2 * j2) | ((2 * i2) << 16), (i2 * hq + j2) * p.k_pad);
@@ -172,14 +182,14 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
             int tm = item;
             if (p.tiles_n > 1) tm = item / p.tiles_n;
-            const int n = tm / p.tiles_per_img;
-            const int p0 = (tm - n * p.tiles_per_img) * p.TH;
+            int n, p0, q0;
+            tile_origin(p, tm, n, p0, q0);
             for (int cb = 0; cb < p.cblks; ++cb) {
                 ok = __all_sync(0xffffffffu, mbar_wait(pempty(ps), pphase ^ 1u, abort_flag, p.status));
                 if (!ok) break;
                 if (elect_one()) {
                     mbar_expect_tx(pfull(ps), (uint32_t)p.patch_box_bytes);
-                    tma_load_4d(patch0 + (uint32_t)ps * p.patch_bytes, &tm_x, pfull(ps), cb * 64, -p.pad_w, p0 - p.pad, n);
+                    tma_load_4d(patch0 + (uint32_t)ps * p.patch_bytes, &tm_x, pfull(ps), cb * 64, q0 - p.pad_w, p0 - p.pad, n);
                 }
                 __syncwarp();
                 if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; }
@@ -287,7 +297,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const float act_lo = p.act == CPRUNE_ACT_NONE ? -INFINITY : 0.f, act_hi = p.act == CPRUNE_ACT_RELU6 ? 6.f : INFINITY;
         const bool store_thread = warp == PK_FIRST_EPI && lane == 0;
         const int groups = (p.FT + 63) / 64;
-        const int n_entries = p.pool ? (p.TH >> 1) * (p.Q >> 1) : 128 * p.MT;
+        const int n_entries = p.pool == 1 ? (p.TH >> 1) * (p.Q >> 1) : ((p.TH - 1) >> 1) * ((p.TW - 1) >> 1);
         // The residual of a group arrives by TMA in the staging buffer the group will use (same box as the store:
         // wrap-around slots read as zero); the values are added there in place.  The load for the next group is
         // issued as soon as its buffer is free.
@@ -295,22 +305,22 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         auto load_residual = [&](int item_, int g_, uint32_t counter) {
             int tm_ = item_, nt_ = 0;
             if (p.tiles_n > 1) { tm_ = item_ / p.tiles_n; nt_ = item_ - tm_ * p.tiles_n; }
-            const int n_ = tm_ / p.tiles_per_img;
-            const int p0_ = (tm_ - n_ * p.tiles_per_img) * p.TH;
+            int n_, p0_, q0_;
+            tile_origin(p, tm_, n_, p0_, q0_);
             const uint32_t b = p.staging_bufs == 2 ? (counter & 1u) : 0u;
             mbar_expect_tx(res_full(b), (uint32_t)(p.TH * p.Wp * 128));
-            tma_load_4d(staging0 + b * stage_buf_bytes, &tm_res, res_full(b), nt_ * p.FT + g_ * 64, 0, p0_, n_);
+            tma_load_4d(staging0 + b * stage_buf_bytes, &tm_res, res_full(b), nt_ * p.FT + g_ * 64, q0_, p0_, n_);
         };
         if (with_res && store_thread && (int)blockIdx.x < total_items) load_residual(blockIdx.x, 0, 0);
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
             int tm = item, nt = 0;
             if (p.tiles_n > 1) { tm = item / p.tiles_n; nt = item - tm * p.tiles_n; }
-            const int n = tm / p.tiles_per_img;
-            const int p0 = (tm - n * p.tiles_per_img) * p.TH;
+            int n, p0, q0;
+            tile_origin(p, tm, n, p0, q0);
             const int k0 = nt * p.FT;
             const int rows_valid = p.P - p0;                 // tile rows below this are real image rows
-            const size_t in_tile = ((size_t)n * p.P + p0) * p.Q * p.k_pad;
-            __nv_bfloat16 *ytile = p.pool ? p.y + ((size_t)n * (p.P >> 1) + (p0 >> 1)) * (p.Q >> 1) * p.k_pad : p.y + in_tile;
+            // first pooled pixel of the tile (2x2 pool: full-width tiles from an even row)
+            __nv_bfloat16 *ytile = p.pool == 1 ? p.y + ((size_t)n * (p.P >> 1) + (p0 >> 1)) * (p.Q >> 1) * p.k_pad : nullptr;
             ok = __all_sync(0xffffffffu, mbar_wait(tfull(acc), acc_phase, abort_flag, p.status, false));
             if (!ok) break;
             tc_fence_after();
@@ -378,7 +388,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     ok = epi_sync();
                     if (!ok) break;
                     if (store_thread) {
-                        if (k0 + g * 64 < p.k_pad) tma_store_4d(&tm_y, staging0 + boff, k0 + g * 64, 0, p0, n);
+                        if (k0 + g * 64 < p.k_pad) tma_store_4d(&tm_y, staging0 + boff, k0 + g * 64, q0, p0, n);
                         tma_store_commit();
                         if (p.staging_bufs == 1) tma_store_wait_read<0>();
                         if (with_res) {
@@ -400,15 +410,46 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (!ok) break;
                 // copy-out: eight threads per output pixel, 16 bytes each
                 const int kg = k0 + g * 64;
-                for (int e = etid; e < n_entries * 8; e += 256) {
-                    const int2 l = lut[e >> 3];
-                    const int chunk = e & 7;
-                    if (l.x >= 0 && (l.x >> 16) < rows_valid && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
-                        const int slot = l.x & 0xffff;
-                        auto staged = [&](int sl) { return *(const uint4 *)(buf + (sl >> 7) * PK_BLOCK_BYTES + sub_off(sl & 127, chunk)); };
-                        uint4 val = bf16x8_max(staged(slot), staged(slot + 1));
-                        val = bf16x8_max(val, bf16x8_max(staged(slot + p.Wp), staged(slot + p.Wp + 1)));
-                        *(uint4 *)(ytile + l.y + kg + chunk * 8) = val;
+                auto staged = [&](int sl, int chunk) { return *(const uint4 *)(buf + (sl >> 7) * PK_BLOCK_BYTES + sub_off(sl & 127, chunk)); };
+                if (p.pool == 1) {
+                    for (int e = etid; e < n_entries * 8; e += 256) {
+                        const int2 l = lut[e >> 3];
+                        const int chunk = e & 7;
+                        if (l.x >= 0 && (l.x >> 16) < rows_valid && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
+                            const int slot = l.x & 0xffff;
+                            uint4 val = bf16x8_max(staged(slot, chunk), staged(slot + 1, chunk));
+                            val = bf16x8_max(val, bf16x8_max(staged(slot + p.Wp, chunk), staged(slot + p.Wp + 1, chunk)));
+                            *(uint4 *)(ytile + l.y + kg + chunk * 8) = val;
+                        }
+                    }
+                } else {
+                    // 3x3 stride-2 windows: the tile computed conv rows p0 .. p0 + TH - 1 (p0 odd or -1) and holds the
+                    // windows of (TH - 1) / 2 x (TW - 1) / 2 pooled pixels.  All nine slots of a window are inside the
+                    // staged tile, so they are loaded unconditionally; conv pixels outside the image are replaced by
+                    // -inf (they never win).
+                    const int tpc = (p.TW - 1) >> 1;
+                    const int pr0 = (p0 + 1) >> 1, pc0 = (q0 + 1) >> 1;
+                    const uint4 ninf = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+                    for (int e = etid; e < n_entries * 8; e += 256) {
+                        const int ent = e >> 3, chunk = e & 7;
+                        const int pi = ent / tpc, pj = ent - pi * tpc;
+                        const int pr = pr0 + pi, pc = pc0 + pj;
+                        if (pr < p.out_h && pc < p.out_w && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
+                            const int r0 = p0 + 2 * pi, c0 = q0 + 2 * pj, s0 = 2 * pi * p.Wp + 2 * pj;
+                            uint4 w[9];
+#pragma unroll
+                            for (int di = 0; di < 3; ++di)
+#pragma unroll
+                                for (int dj = 0; dj < 3; ++dj) {
+                                    const bool inside = r0 + di >= 0 && r0 + di < p.P && c0 + dj >= 0 && c0 + dj < p.Q;
+                                    const uint4 t = staged(s0 + di * p.Wp + dj, chunk);
+                                    w[di * 3 + dj] = inside ? t : ninf;
+                                }
+                            const uint4 a0 = bf16x8_max(bf16x8_max(w[0], w[1]), bf16x8_max(w[2], w[3]));
+                            const uint4 a1 = bf16x8_max(bf16x8_max(w[4], w[5]), bf16x8_max(w[6], w[7]));
+                            *(uint4 *)(p.y + (((size_t)n * p.out_h + pr) * p.out_w + pc) * p.k_pad + kg + chunk * 8) =
+                                bf16x8_max(bf16x8_max(a0, a1), w[8]);
+                        }
                     }
                 }
                 if (p.staging_bufs == 1) {
@@ -506,7 +547,10 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     if (!patch_geometry(i, &g)) return CPRUNE_ERR_UNSUPPORTED;
     const int Wp = g.Wp;
     const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
+    const bool pool3 = plan->opts.pool == CPRUNE_POOL_MAX3X3S2;
     if (pool && (plan->opts.residual || (i.P & 1) || (i.Q & 1))) return CPRUNE_ERR_UNSUPPORTED;
+    // the 3x3 pool needs tiles narrower than the image, which only tasks without wrap-around slots allow
+    if (pool3 && (plan->opts.residual || g.kS != 1)) return CPRUNE_ERR_UNSUPPORTED;
     const int k16 = round_up(i.K, 16);
     const int cblks = g.cblks, ksteps_last = g.ksteps_last, RB = 128;
     const int RS = g.kR * g.kS;
@@ -516,11 +560,27 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     const char *force_tn = getenv("CPRUNE_PATCH_TN");
     for (int MT = 1; MT <= 2; ++MT) {
         if (force_mt && atoi(force_mt) != MT) continue;
-        int TH = (128 * MT) / Wp;
-        if (TH > i.P) TH = i.P;
-        if (pool) TH &= ~1;
-        if (TH < 1) continue;
-        const int tiles_per_img = (i.P + TH - 1) / TH;
+      // candidate tile shapes: whole-width rows; for the 3x3 pool (2 tpr + 1) x (2 tpc + 1) conv pixels around tpr x tpc pooled ones
+      const int n_shapes = pool3 ? 32 * 32 : 1;
+      for (int shape = 0; shape < n_shapes; ++shape) {
+        int TH, TW = i.Q, tiles_w = 1, step_h, step_w = i.Q, org = 0, tiles_per_img, Wp = g.Wp;
+        if (pool3) {
+            const int tpr = shape / 32 + 1, tpc = shape % 32 + 1;
+            if (tpr > i.out_h || tpc > i.out_w) continue;
+            TH = 2 * tpr + 1; TW = 2 * tpc + 1;
+            if (TH * TW > 128 * MT) continue;
+            Wp = TW;
+            step_h = 2 * tpr; step_w = 2 * tpc; org = -1;
+            tiles_w = (i.out_w + tpc - 1) / tpc;
+            tiles_per_img = ((i.out_h + tpr - 1) / tpr) * tiles_w;
+        } else {
+            TH = (128 * MT) / Wp;
+            if (TH > i.P) TH = i.P;
+            if (pool) TH &= ~1;
+            if (TH < 1) continue;
+            step_h = TH;
+            tiles_per_img = (i.P + TH - 1) / TH;
+        }
         for (int tiles_n = 1; tiles_n <= 8; ++tiles_n) {
             if (force_tn && atoi(force_tn) != tiles_n) continue;
             // with several filter tiles every tile ends on a 64-filter boundary: the stores are 64 filters wide and
@@ -557,9 +617,10 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             if (resident) t += RS * cblks * FT;    // one-time filter load
             if (t < best) {
                 best = t;
-                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes};
+                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org};
             }
         }
+      }
     }
     if (best >= 1e30) return CPRUNE_ERR_UNSUPPORTED;
     // share of accumulator rows that hold real pixels; below one half the im2col kernel is the better choice
@@ -577,7 +638,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     plan->ipp = 0;
     plan->partial_bytes = 0;
     plan->pre_bytes = g.stem ? ((size_t)i.N * g.He * g.WP * 32 + 255) / 256 * 256 : 0;
-    plan->fused_pool = pool ? 1 : 0;
+    plan->fused_pool = (pool || pool3) ? 1 : 0;
     i.tile_m = 128 * bt.MT;
     i.tile_n = bt.FT;
     i.tile_k = 64;
@@ -592,34 +653,39 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     return CPRUNE_OK;
 }
 
-// Regroups a bf16 NHWC tensor with c_pad = 8 channels (C real ones) into 16-channel pixels, one per sf x sf block of
-// input pixels, in rows of WP pixels of which the first pad_lo (and whatever follows the image) are zero:
-// out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
-__global__ void __launch_bounds__(256) regroup_kernel(const bf16x8 *__restrict__ x, int N, int H, int W, int C, int sf, int pad_lo,
-                                                      int WP, uint4 *__restrict__ out) {
+// Regroups an NHWC tensor with C channels per pixel (T = bf16 with 8 channel lanes in memory, or float32 with C) into
+// 16-channel bf16 pixels, one per sf x sf block of input pixels, in rows of WP pixels of which the first pad_lo (and
+// whatever follows the image) are zero:
+//   out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
+// Eight threads per output pixel, two channels each: the 32 bytes of a pixel are written by neighbouring lanes.
+template <typename T>
+__global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, int N, int H, int W, int C, int c_mem, int sf, int pad_lo,
+                                                      int WP, __nv_bfloat162 *__restrict__ out) {
     pdl_trigger();
     pdl_wait();
     const int H2 = H / sf, W2 = W / sf;
-    const long long total = (long long)N * H2 * WP;
+    const long long total = (long long)N * H2 * WP * 8;
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-        const int wp = (int)(e % WP);
-        const long long t = e / WP;
+        const int pair = (int)(e & 7);
+        const long long px = e >> 3;
+        const int wp = (int)(px % WP);
+        const long long t = px / WP;
         const int h2 = (int)(t % H2);
         const long long n = t / H2;
         const int w2 = wp - pad_lo;
-        __align__(16) __nv_bfloat16 o[16];
-#pragma unroll
-        for (int c = 0; c < 16; ++c) o[c] = __float2bfloat16_rn(0.f);
+        float v[2] = {0.f, 0.f};
         if (w2 >= 0 && w2 < W2) {
-            for (int dy = 0; dy < sf; ++dy)
-                for (int dx = 0; dx < sf; ++dx) {
-                    const bf16x8 v = ldg8(x + (n * H + sf * h2 + dy) * W + sf * w2 + dx);
-                    const __nv_bfloat16 *pv = reinterpret_cast<const __nv_bfloat16 *>(&v);
-                    for (int c = 0; c < C; ++c) o[(dy * sf + dx) * C + c] = pv[c];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int ch = 2 * pair + k;
+                const int blk = ch / C, c = ch - blk * C;
+                if (blk < sf * sf) {
+                    const int dy = blk / sf, dx = blk - dy * sf;
+                    v[k] = (float)x[((n * H + sf * h2 + dy) * W + sf * w2 + dx) * c_mem + c];
                 }
+            }
         }
-        out[2 * e] = *reinterpret_cast<const uint4 *>(o);
-        out[2 * e + 1] = *reinterpret_cast<const uint4 *>(o + 8);
+        out[e] = __floats2bfloat162_rn(v[0], v[1]);
     }
 }
 
@@ -665,21 +731,36 @@ size_t packed_weight_bytes_patch(const cprune_plan *plan) {
     return (size_t)i.k_alloc * g.Re * g.Se * 32;
 }
 
+cprune_status regroup_stem_input(const cprune_plan *plan, const void *x, int x_is_f32, void *scratch, cudaStream_t st) {
+    const cprune_plan_info &i = plan->info;
+    PatchGeometry g;
+    if (!patch_geometry(i, &g) || !g.stem || !x || !scratch) return CPRUNE_ERR_INVALID_ARG;
+    const long long total = (long long)i.N * g.He * g.WP * 8;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (x_is_f32)
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3((unsigned)blocks), dim3(256), 0, st, (const float *)x, i.N, i.H, i.W, i.C, i.C,
+                                         g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
+    else
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(256), 0, st, (const __nv_bfloat16 *)x, i.N,
+                                         i.H, i.W, i.C, i.c_pad, g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
+    return CPRUNE_OK;
+}
+
 cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res, void *y,
-                                void *scratch, cudaStream_t st) {
+                                void *scratch, cudaStream_t st, bool input_regrouped) {
     const cprune_plan_info &i = plan->info;
     const PatchTiling &t = plan->pt;
     PatchGeometry g;
     if (!patch_geometry(i, &g)) return CPRUNE_ERR_INTERNAL;
-    const int Wp = g.Wp;
+    const int Wp = t.TW + g.kS - 1;    // patch row pitch: the tile's width plus the filter's
     const void *xe = x;        // the tensor the patch loads read
     if (g.stem) {
         if (!scratch) return CPRUNE_ERR_INVALID_ARG;
-        const long long total = (long long)i.N * g.He * g.WP;
-        long long blocks = (total + 255) / 256;
-        if (blocks > 148 * 16) blocks = 148 * 16;
-        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel, dim3((unsigned)blocks), dim3(256), 0, st, (const bf16x8 *)x, i.N, i.H, i.W, i.C, g.sf, g.pad_lo,
-                                         g.WP, (uint4 *)scratch));
+        if (!input_regrouped) {
+            cprune_status rs = regroup_stem_input(plan, x, 0, scratch, st);
+            if (rs != CPRUNE_OK) return rs;
+        }
         xe = scratch;
     }
     CUtensorMap tm_x, tm_w, tm_y, tm_res;
@@ -753,13 +834,15 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     }
     PatchParams p;
     p.P = i.P; p.Q = i.Q; p.Wp = Wp; p.TH = t.TH; p.tiles_per_img = t.tiles_per_img;
+    p.TW = t.TW; p.tiles_w = t.tiles_w; p.step_h = t.step_h; p.step_w = t.step_w; p.org = t.org;
+    p.out_h = i.out_h; p.out_w = i.out_w;
     p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.FT = t.FT; p.MT = t.MT; p.R = g.kR; p.S = g.kS; p.pad = g.pad_lo; p.pad_w = g.pad_w;
     p.cblks = g.cblks;
     p.ksteps_last = g.ksteps_last;
     p.k_pad = i.k_pad;
     p.act = plan->opts.activation;
     p.wstages = t.wstages; p.resident = t.resident; p.acc_bufs = t.acc_bufs; p.staging_bufs = t.staging_bufs;
-    p.pool = plan->fused_pool;
+    p.pool = plan->fused_pool ? plan->opts.pool : 0;
     p.patch_bytes = t.patch_bytes;
     p.patch_box_bytes = Wp * (t.TH + g.kR - 1) * 128;
     p.rb16 = 8;

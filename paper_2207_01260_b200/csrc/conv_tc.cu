@@ -979,9 +979,9 @@ static int sm_count() {
 }
 
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
-                                 void *y, void *partial, cudaStream_t st) {
+                                 void *y, void *partial, cudaStream_t st, bool input_regrouped) {
     const cprune_plan_info &i = plan->info;
-    if (plan->patch) return launch_conv_patch(plan, x, w, b, res, y, partial, st);
+    if (plan->patch) return launch_conv_patch(plan, x, w, b, res, y, partial, st, input_regrouped);
     CUtensorMap tm_x, tm_w, tm_y, tm_res, tm_id;
     const bool split = plan->splits > 1;
     if (split && !partial) return CPRUNE_ERR_INVALID_ARG;

@@ -59,8 +59,21 @@ static cprune_status enqueue(cprune_model *m, const float *x, float *logits, cud
     return s;
 }
 
+// True when the model's input is read by its first task only and that task is a stem that works on a regrouped
+// input: the float32 image is then cast and regrouped in one pass and the bf16 NHWC copy is never written.
+static bool stem_reads_image_directly(const cprune_model *m) {
+    if (m->tasks.empty()) return false;
+    const cprune_task_desc &d0 = m->tasks[0];
+    if (d0.op != CPRUNE_OP_CONV || d0.in != 0 || !d0.plan || !d0.plan->patch || !d0.plan->narrow) return false;
+    for (size_t t = 1; t < m->tasks.size(); ++t)
+        if (m->tasks[t].in == 0 || m->tasks[t].res == 0) return false;
+    return true;
+}
+
 static cprune_status enqueue_chain(cprune_model *m, const float *x, float *logits, cudaStream_t st) {
-    cprune_status s = cprune_cast_input(x, (size_t)m->N * m->H * m->W, m->C, tensor_ptr(m, 0), st);
+    const bool direct = stem_reads_image_directly(m);
+    cprune_status s = direct ? regroup_stem_input(m->tasks[0].plan, x, 1, stem_scratch(m->tasks[0].plan, m->workspace), st)
+                             : cprune_cast_input(x, (size_t)m->N * m->H * m->W, m->C, tensor_ptr(m, 0), st);
     if (s != CPRUNE_OK) return s;
     for (size_t t = 0; t < m->tasks.size(); ++t) {
         const cprune_task_desc &d = m->tasks[t];
@@ -70,8 +83,8 @@ static cprune_status enqueue_chain(cprune_model *m, const float *x, float *logit
         void *pout = last ? (void *)logits : tensor_ptr(m, d.out);
         switch (d.op) {
             case CPRUNE_OP_CONV:
-                s = cprune_task_run(d.plan, pin, d.w, d.b, d.res >= 0 ? tensor_ptr(m, d.res) : nullptr, pout,
-                                    m->workspace, st);
+                s = task_run_internal(d.plan, pin, d.w, d.b, d.res >= 0 ? tensor_ptr(m, d.res) : nullptr, pout, m->workspace, st,
+                                      t == 0 && direct);
                 break;
             case CPRUNE_OP_MAXPOOL:
                 s = cprune_maxpool(pin, in.n, in.h, in.w, in.c, d.p0, d.p1, d.p2, pout, st);
@@ -132,7 +145,8 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
                 }
                 o.h = i.out_h; o.w = i.out_w; o.c = i.K;
                 if (i.workspace_bytes > m->workspace_bytes) m->workspace_bytes = i.workspace_bytes;
-                m->launches += ((d.plan->opts.pool && !(i.kernel == CPRUNE_KERNEL_TENSOR && d.plan->fused_pool)) ? 2 : 1) + (d.plan->splits > 1 ? 1 : 0);
+                m->launches += ((d.plan->opts.pool && !(i.kernel == CPRUNE_KERNEL_TENSOR && d.plan->fused_pool)) ? 2 : 1) + (d.plan->splits > 1 ? 1 : 0) +
+                               ((d.plan->patch && d.plan->narrow) ? 1 : 0);
                 break;
             }
             case CPRUNE_OP_MAXPOOL:
@@ -162,6 +176,7 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
         m->tensors[d.out] = o;
     }
     if (st != CPRUNE_OK) { delete m; return st; }
+    if (stem_reads_image_directly(m)) m->launches -= 1;     // one pass casts and regroups the image
     size_t off = 0;
     for (auto &kv : m->tensors) {
         kv.second.bytes = (size_t)kv.second.n * kv.second.h * kv.second.w * kv.second.c_pad * 2;

@@ -43,6 +43,7 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     i.Q = (i.W + 2 * i.pad - i.S) / i.stride + 1;
     i.out_h = i.P; i.out_w = i.Q;
     if (pl->opts.pool == CPRUNE_POOL_MAX2X2) { i.out_h = i.P / 2; i.out_w = i.Q / 2; }
+    if (pl->opts.pool == CPRUNE_POOL_MAX3X3S2) { i.out_h = (i.P - 1) / 2 + 1; i.out_w = (i.Q - 1) / 2 + 1; }
     i.c_pad = cprune_padded_channels(i.C);
     i.k_pad = cprune_padded_channels(i.K);
     i.k_alloc = i.k_pad;
@@ -76,13 +77,14 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     }
     if (st != CPRUNE_OK) { delete pl; return st; }
     i.kernel = family;
+    i.variant = (family == CPRUNE_KERNEL_TENSOR && pl->patch) ? 1 : 0;
     const double rs = (double)i.R * i.S;
     const int s_packed = (family == CPRUNE_KERNEL_TENSOR && pl->s_packed > 0) ? pl->s_packed : i.S;
     i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * s_packed * i.c_pad * 2;
     if (family == CPRUNE_KERNEL_TENSOR && pl->patch && pl->narrow) i.packed_weight_bytes = packed_weight_bytes_patch(pl);
     i.packed_bias_bytes = (size_t)i.k_alloc * sizeof(float);
     // workspace: [unpooled conv output if a pool follows][split-K partial sums]
-    const bool separate_pool = pl->opts.pool == CPRUNE_POOL_MAX2X2 && !(family == CPRUNE_KERNEL_TENSOR && pl->fused_pool);
+    const bool separate_pool = pl->opts.pool != CPRUNE_POOL_NONE && !(family == CPRUNE_KERNEL_TENSOR && pl->fused_pool);
     pl->pool_bytes = separate_pool ? ((size_t)i.N * i.P * i.Q * i.k_pad * 2 + 255) / 256 * 256 : 0;
     // (patch kernel on a regrouped stem: the regrouped input takes the place of the partial sums)
     i.workspace_bytes = pl->pool_bytes + (family == CPRUNE_KERNEL_TENSOR ? pl->partial_bytes + pl->pre_bytes : 0);
@@ -90,6 +92,33 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
                                  (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
                                  (double)i.K * (i.C / i.groups) * rs) + 4.0 * i.K;
     *out = pl;
+    return CPRUNE_OK;
+}
+
+
+cprune_status task_run_internal(cprune_plan *plan, const void *x, const void *w_packed, const float *b_packed, const void *residual,
+                                void *y, void *workspace, cudaStream_t st, bool input_regrouped) {
+    if (!plan || !x || !w_packed || !b_packed || !y) return CPRUNE_ERR_INVALID_ARG;
+    if ((plan->opts.residual != 0) != (residual != nullptr)) return CPRUNE_ERR_INVALID_ARG;
+    if (((uintptr_t)x | (uintptr_t)w_packed | (uintptr_t)y | (uintptr_t)residual | (uintptr_t)workspace) & 15)
+        return CPRUNE_ERR_INVALID_ARG;
+    const cprune_plan_info &i = plan->info;
+    const bool pool = plan->opts.pool != CPRUNE_POOL_NONE && !(i.kernel == CPRUNE_KERNEL_TENSOR && plan->fused_pool);
+    if (i.workspace_bytes && !workspace) return CPRUNE_ERR_INVALID_ARG;
+    void *conv_out = pool ? workspace : y;
+    void *partial = (plan->partial_bytes || plan->pre_bytes) ? (void *)((char *)workspace + plan->pool_bytes) : nullptr;
+    cprune_status s;
+    switch (i.kernel) {
+        case CPRUNE_KERNEL_TENSOR: s = launch_conv_tensor(plan, x, w_packed, b_packed, residual, conv_out, partial, st, input_regrouped); break;
+        case CPRUNE_KERNEL_DIRECT: s = launch_conv_direct(plan, x, w_packed, b_packed, residual, conv_out, st); break;
+        case CPRUNE_KERNEL_DEPTHWISE: s = launch_depthwise(plan, x, w_packed, b_packed, residual, conv_out, st); break;
+        default: return CPRUNE_ERR_INTERNAL;
+    }
+    if (s != CPRUNE_OK) return s;
+    if (pool) {
+        if (plan->opts.pool == CPRUNE_POOL_MAX3X3S2) return launch_maxpool(conv_out, i.N, i.P, i.Q, i.k_pad, 3, 2, 1, y, st);
+        return launch_maxpool(conv_out, i.N, i.P, i.Q, i.k_pad, 2, 2, 0, y, st);
+    }
     return CPRUNE_OK;
 }
 
@@ -108,7 +137,7 @@ cprune_status cprune_task_plan(int N, int C, int H, int W, int K, int R, int S, 
     if (H + 2 * pad < R || W + 2 * pad < S) return CPRUNE_ERR_INVALID_ARG;
     cprune_task_opts o = {CPRUNE_ACT_RELU, 0, CPRUNE_POOL_NONE, CPRUNE_KERNEL_AUTO};
     if (opts) o = *opts;
-    if (o.activation < 0 || o.activation > 2 || o.pool < 0 || o.pool > 1 || o.kernel < 0 || o.kernel > 3 ||
+    if (o.activation < 0 || o.activation > 2 || o.pool < 0 || o.pool > 2 || o.kernel < 0 || o.kernel > 3 ||
         (o.residual != 0 && o.residual != 1))
         return CPRUNE_ERR_INVALID_ARG;
     if (groups != 1) {
@@ -177,26 +206,7 @@ cprune_status cprune_cache_stats(int *n_plans, long long *n_hits) {
 
 cprune_status cprune_task_run(cprune_plan *plan, const void *x, const void *w_packed, const float *b_packed,
                               const void *residual, void *y, void *workspace, void *stream) {
-    if (!plan || !x || !w_packed || !b_packed || !y) return CPRUNE_ERR_INVALID_ARG;
-    if ((plan->opts.residual != 0) != (residual != nullptr)) return CPRUNE_ERR_INVALID_ARG;
-    if (((uintptr_t)x | (uintptr_t)w_packed | (uintptr_t)y | (uintptr_t)residual | (uintptr_t)workspace) & 15)
-        return CPRUNE_ERR_INVALID_ARG;
-    const cprune_plan_info &i = plan->info;
-    const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2 && !(i.kernel == CPRUNE_KERNEL_TENSOR && plan->fused_pool);
-    if (i.workspace_bytes && !workspace) return CPRUNE_ERR_INVALID_ARG;
-    void *conv_out = pool ? workspace : y;
-    void *partial = (plan->partial_bytes || plan->pre_bytes) ? (void *)((char *)workspace + plan->pool_bytes) : nullptr;
-    cudaStream_t st = (cudaStream_t)stream;
-    cprune_status s;
-    switch (i.kernel) {
-        case CPRUNE_KERNEL_TENSOR: s = launch_conv_tensor(plan, x, w_packed, b_packed, residual, conv_out, partial, st); break;
-        case CPRUNE_KERNEL_DIRECT: s = launch_conv_direct(plan, x, w_packed, b_packed, residual, conv_out, st); break;
-        case CPRUNE_KERNEL_DEPTHWISE: s = launch_depthwise(plan, x, w_packed, b_packed, residual, conv_out, st); break;
-        default: return CPRUNE_ERR_INTERNAL;
-    }
-    if (s != CPRUNE_OK) return s;
-    if (pool) return launch_maxpool(conv_out, i.N, i.P, i.Q, i.k_pad, 2, 2, 0, y, st);
-    return CPRUNE_OK;
+    return task_run_internal(plan, x, w_packed, b_packed, residual, y, workspace, (cudaStream_t)stream, false);
 }
 
 }  // extern "C"

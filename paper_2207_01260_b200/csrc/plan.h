@@ -13,6 +13,7 @@
 // rows, FT filters.
 struct PatchTiling {
     int MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes;
+    int TW, tiles_w, step_h, step_w, org;   // tile width, tiles per image row, distance between tiles, origin offset
 };
 
 struct cprune_plan {
@@ -58,11 +59,19 @@ cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, 
 // tcgen05 implicit GEMM
 cprune_status plan_conv_tensor(cprune_plan *plan);  // fills tile fields of plan->info; UNSUPPORTED if not eligible
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
-                                 void *y, void *partial, cudaStream_t st);
+                                 void *y, void *partial, cudaStream_t st, bool input_regrouped = false);
 // stride-1 R x S > 1 tasks with the input patch resident in shared memory (part of the tensor family)
 cprune_status plan_conv_patch(cprune_plan *plan);   // UNSUPPORTED if the task is not eligible or would waste the tile
 cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,
-                                void *y, void *scratch, cudaStream_t st);
+                                void *y, void *scratch, cudaStream_t st, bool input_regrouped = false);
+// regrouped 16-channel input of a stem plan (plan->narrow) written to `scratch` from the benchmark's bf16 input or straight
+// from the float32 image (cast and regrouping in one pass)
+cprune_status regroup_stem_input(const cprune_plan *plan, const void *x, int x_is_f32, void *scratch, cudaStream_t st);
+// cprune_task_run with one more option: the regrouped input of a stem plan is already in the workspace
+cprune_status task_run_internal(cprune_plan *plan, const void *x, const void *w_packed, const float *b_packed, const void *residual,
+                                void *y, void *workspace, cudaStream_t st, bool input_regrouped);
+// where in a task's workspace the regrouped stem input lives
+inline void *stem_scratch(const cprune_plan *plan, void *workspace) { return (char *)workspace + plan->pool_bytes; }
 // filters of a regrouped stem (plan->narrow) and their size
 cprune_status pack_conv_patch(const cprune_plan *plan, const float *w, void *w_packed, cudaStream_t st);
 size_t packed_weight_bytes_patch(const cprune_plan *plan);

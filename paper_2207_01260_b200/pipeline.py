@@ -18,9 +18,10 @@ from . import binding as B
 
 
 class PrunedNetwork:
-    def __init__(self, table: dict, weights: dict, batch: int, device="cuda:0", kernel="auto"):
+    def __init__(self, table: dict, weights: dict, batch: int, device="cuda:0", kernel="auto", fuse_pool=True):
         self.table, self.batch, self.device = table, batch, torch.device(device)
         self.kernel = kernel
+        self.fuse_pool = fuse_pool
         self.params = {k: (torch.from_numpy(np.ascontiguousarray(w)).to(self.device),
                            torch.from_numpy(np.ascontiguousarray(b)).to(self.device)) for k, (w, b) in weights.items()}
         self.kept = {}
@@ -80,29 +81,51 @@ class PrunedNetwork:
                 ids[name] = len(ids)
             return ids[name]
 
+        # A 3x3 stride-2 pad-1 max-pool that is the only reader of a conv task's output becomes that task's pool
+        # option: the unpooled tensor is then never stored.
+        layers = self.table["layers"]
+        readers = {}
+        for l in layers:
+            for key in ("in", "res"):
+                if l.get(key) is not None:
+                    readers.setdefault(l[key], []).append(l["name"])
+        fused = {}      # conv name -> the pool layer it absorbs
+        if self.fuse_pool:
+            for a, b in zip(layers, layers[1:]):
+                if (a["kind"] == "conv" and b["kind"] == "maxpool" and b["in"] == a["out"] and a.get("pool") is None
+                        and a.get("res") is None and (b["k"], b["stride"], b["pad"]) == (3, 2, 1)
+                        and readers.get(a["out"]) == [b["name"]]):
+                    fused[a["name"]] = b
+        absorbed = {b["name"] for b in fused.values()}
+        self.fused_pools, self.absorbed = fused, absorbed
+
         for l in self.table["layers"]:
             kind = l["kind"]
+            if l["name"] in absorbed:
+                continue
             h, w, c = shape[l["in"]]
             if kind == "flatten":
                 ids[l["out"]] = ids[l["in"]]
                 shape[l["out"]] = shape[l["in"]]
                 continue
             d = B.TaskDesc()
-            d.in_, d.out, d.res = tid(l["in"]), tid(l["out"]), -1
+            out_name = fused[l["name"]]["out"] if l["name"] in fused else l["out"]
+            d.in_, d.out, d.res = tid(l["in"]), tid(out_name), -1
             if kind == "conv":
                 wt, bs = self.params[l["name"]]
                 K, cg = wt.shape[0], wt.shape[1]
                 groups = K if l["groups"] > 1 else 1
                 assert cg * groups == c, (l["name"], cg, groups, c)
                 plan = B.cprune_task_plan(self.batch, c, h, w, K, l["R"], l["S"], l["stride"], l["pad"], groups,
-                                          l["act"], l.get("res") is not None, l.get("pool"),
+                                          l["act"], l.get("res") is not None,
+                                          "max3x3s2" if l["name"] in fused else l.get("pool"),
                                           self.kernel if groups == 1 else "auto")
                 wp, bp = B.cprune_pack_weights(plan, wt, bs)
                 self.plans[l["name"]], self.packed[l["name"]] = plan, (wp, bp)
                 d.op, d.plan, d.w, d.b = B.OP_CONV, plan.handle, wp.data_ptr(), bp.data_ptr()
                 if l.get("res") is not None:
                     d.res = tid(l["res"])
-                shape[l["out"]] = (plan.out_h, plan.out_w, K)
+                shape[out_name] = (plan.out_h, plan.out_w, K)
             elif kind == "maxpool":
                 d.op, d.p0, d.p1, d.p2 = B.OP_MAXPOOL, l["k"], l["stride"], l["pad"]
                 shape[l["out"]] = ((h + 2 * l["pad"] - l["k"]) // l["stride"] + 1,

@@ -40,7 +40,10 @@ def check_task(cp, N, C, H, W, K, R, stride, pad, groups=1, act="relu", with_res
     x, w, b, res = wl.conv_task_tensors(seed, N, C, H, W, K, R, R, groups, with_res, P, Q)
     y, plan = run_task(cp, x, w, b, stride, pad, groups, act, res, pool, kernel)
     ref, bound = oracle.conv2d(x, w, b, stride, pad, groups, act, res, with_bound=True)
-    if pool:
+    if pool == "max3x3s2":
+        # the error bound of a maximum is at most the largest bound in its window
+        ref, bound = oracle.maxpool(ref, 3, 2, 1), oracle.maxpool(bound, 3, 2, 1)
+    elif pool:
         ref, bound = oracle.maxpool(ref, 2, 2, 0), oracle.maxpool(bound, 2, 2, 0)
     assert y.shape == (N, plan.out_h, plan.out_w, plan.k_pad)
     assert np.all(y[..., K:] == 0), "pad lanes must be written as zero"
@@ -165,6 +168,27 @@ def test_dense_task_epilogues(cp, kernel):
 def test_fused_maxpool(cp, case):
     N, C, HW, K = case
     check_task(cp, N, C, HW, HW, K, 3, 1, 1, act="relu", pool="max2x2", kernel="tensor")
+
+
+def test_stems_on_the_patch_kernel(cp):
+    # enough tiles for the patch kernel: the input is regrouped into 16-channel pixels (stride 1 and 2)
+    plan = check_task(cp, 16, 3, 64, 64, 64, 7, 2, 3, kernel="tensor")
+    assert plan.variant == 1 and plan.workspace_bytes > 0     # the workspace holds the regrouped input
+    check_task(cp, 16, 3, 62, 60, 32, 3, 2, 1, act="relu6", kernel="tensor")
+    check_task(cp, 24, 3, 32, 32, 45, 3, 1, 1, kernel="tensor")
+    check_task(cp, 20, 4, 36, 28, 24, 5, 1, 2, act="none", kernel="tensor")
+
+
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, stride, pad: fused in the patch kernel (tiles around whole 3x3 windows, even and odd extents),
+    # and as a separate pass (few tiles; a task with wrap-around slots)
+    (16, 3, 64, 64, 64, 7, 2, 3), (12, 3, 60, 52, 40, 7, 2, 3), (40, 3, 30, 30, 24, 3, 1, 1),
+    (2, 3, 64, 64, 64, 7, 2, 3), (2, 16, 30, 30, 24, 3, 1, 1)])
+def test_maxpool_3x3_stride_2(cp, case):
+    N, C, H, W, K, R, stride, pad = case
+    plan = check_task(cp, N, C, H, W, K, R, stride, pad, act="relu", pool="max3x3s2", kernel="tensor")
+    P = oracle.out_size(H, R, stride, pad)
+    assert plan.out_h == (P - 1) // 2 + 1
 
 
 @pytest.mark.parametrize("C", [64, 65, 66, 67, 68, 69, 70, 71, 72, 73, 79, 80, 81])
@@ -333,7 +357,15 @@ def test_intermediate_activations_match(cp):
     net.run(_dev(x))
     pw, _ = oracle.prune_model(table, weights)
     _, tensors = oracle.model_ref(table, pw, x, matched=True, keep_tensors=True)
-    for name in ("s0", "p0", "l1b1_h", "l1b1_o", "l2b1_id", "l2b1_o", "l4b2_o", "g"):
+    # the stem's 3x3 max-pool is fused into the stem task: its unpooled output "s0" is never stored
+    for name in ("p0", "l1b1_h", "l1b1_o", "l2b1_id", "l2b1_o", "l4b2_o", "g"):
+        got = net.activation(name)
+        ref = tensors[name].reshape(got.shape)
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert rel <= 1e-2, (name, rel)
+    net = PrunedNetwork(table, weights, 2, fuse_pool=False)
+    net.run(_dev(x))
+    for name in ("s0", "p0"):
         got = net.activation(name)
         ref = tensors[name].reshape(got.shape)
         rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
