@@ -659,19 +659,17 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
 //   out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
 // Eight threads per output pixel, two channels each: the 32 bytes of a pixel are written by neighbouring lanes.
 template <typename T>
-__global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, int N, int H, int W, int C, int c_mem, int sf, int pad_lo,
-                                                      int WP, __nv_bfloat162 *__restrict__ out) {
+__global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, int H, int W, int C, int c_mem, int sf, int pad_lo, int WP,
+                                                      __nv_bfloat162 *__restrict__ out) {
     pdl_trigger();
     pdl_wait();
+    // one block per output row (image n, regrouped row h2); no per-element division by anything but C
     const int H2 = H / sf, W2 = W / sf;
-    const long long total = (long long)N * H2 * WP * 8;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-        const int pair = (int)(e & 7);
-        const long long px = e >> 3;
-        const int wp = (int)(px % WP);
-        const long long t = px / WP;
-        const int h2 = (int)(t % H2);
-        const long long n = t / H2;
+    const int n = blockIdx.x / H2, h2 = blockIdx.x - n * H2;
+    const T *rows = x + ((size_t)n * H + (size_t)sf * h2) * W * c_mem;
+    __nv_bfloat162 *orow = out + (size_t)blockIdx.x * WP * 8;
+    for (int e = threadIdx.x; e < WP * 8; e += blockDim.x) {
+        const int pair = e & 7, wp = e >> 3;
         const int w2 = wp - pad_lo;
         float v[2] = {0.f, 0.f};
         if (w2 >= 0 && w2 < W2) {
@@ -681,11 +679,11 @@ __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, i
                 const int blk = ch / C, c = ch - blk * C;
                 if (blk < sf * sf) {
                     const int dy = blk / sf, dx = blk - dy * sf;
-                    v[k] = (float)x[((n * H + sf * h2 + dy) * W + sf * w2 + dx) * c_mem + c];
+                    v[k] = (float)rows[((size_t)dy * W + sf * w2 + dx) * c_mem + c];
                 }
             }
         }
-        out[e] = __floats2bfloat162_rn(v[0], v[1]);
+        orow[e] = __floats2bfloat162_rn(v[0], v[1]);
     }
 }
 
@@ -735,15 +733,13 @@ cprune_status regroup_stem_input(const cprune_plan *plan, const void *x, int x_i
     const cprune_plan_info &i = plan->info;
     PatchGeometry g;
     if (!patch_geometry(i, &g) || !g.stem || !x || !scratch) return CPRUNE_ERR_INVALID_ARG;
-    const long long total = (long long)i.N * g.He * g.WP * 8;
-    long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 64) blocks = 148 * 64;
+    const unsigned blocks = (unsigned)(i.N * g.He);
     if (x_is_f32)
-        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3((unsigned)blocks), dim3(256), 0, st, (const float *)x, i.N, i.H, i.W, i.C, i.C,
-                                         g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3(blocks), dim3(256), 0, st, (const float *)x, i.H, i.W, i.C, i.C, g.sf, g.pad_lo,
+                                         g.WP, (__nv_bfloat162 *)scratch));
     else
-        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(256), 0, st, (const __nv_bfloat16 *)x, i.N,
-                                         i.H, i.W, i.C, i.c_pad, g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16 *)x, i.H, i.W, i.C,
+                                         i.c_pad, g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
     return CPRUNE_OK;
 }
 
