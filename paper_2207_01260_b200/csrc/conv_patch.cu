@@ -518,6 +518,7 @@ static bool patch_geometry(const cprune_plan_info &i, PatchGeometry *g) {
     } else if (i.c_pad == 8 && i.stride <= 2 && i.C * i.stride * i.stride <= 16 && i.R * i.S > 1 && i.R <= 8 && i.S <= 8) {
         const int sf = i.stride;
         if ((i.H % sf) || (i.W % sf)) return false;
+        if ((size_t)sf * i.W * 16 > 48 * 1024) return false;      // the regrouping pass stages sf input rows in shared memory
         if (i.R - 1 - i.pad < 0 || i.S - 1 - i.pad < 0) return false;
         g->stem = 1; g->sf = sf;
         g->pad_lo = sf == 1 ? i.pad : (i.pad + 1) / 2;
@@ -663,10 +664,23 @@ __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, i
                                                       __nv_bfloat162 *__restrict__ out) {
     pdl_trigger();
     pdl_wait();
-    // one block per output row (image n, regrouped row h2); no per-element division by anything but C
+    // one block per output row (image n, regrouped row h2): its sf input rows are contiguous in memory and are
+    // brought into shared memory with 16-byte loads first
+    extern __shared__ __align__(16) unsigned char rg_smem[];
+    T *srow = reinterpret_cast<T *>(rg_smem);
     const int H2 = H / sf, W2 = W / sf;
     const int n = blockIdx.x / H2, h2 = blockIdx.x - n * H2;
     const T *rows = x + ((size_t)n * H + (size_t)sf * h2) * W * c_mem;
+    const int n_elems = sf * W * c_mem;
+    const size_t n_bytes = (size_t)n_elems * sizeof(T);
+    if (((reinterpret_cast<uintptr_t>(rows) | n_bytes) & 15) == 0) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(rows);
+        uint4 *dst = reinterpret_cast<uint4 *>(rg_smem);
+        for (int i = threadIdx.x; i < (int)(n_bytes >> 4); i += blockDim.x) dst[i] = __ldg(src + i);
+    } else {
+        for (int i = threadIdx.x; i < n_elems; i += blockDim.x) srow[i] = rows[i];
+    }
+    __syncthreads();
     __nv_bfloat162 *orow = out + (size_t)blockIdx.x * WP * 8;
     for (int e = threadIdx.x; e < WP * 8; e += blockDim.x) {
         const int pair = e & 7, wp = e >> 3;
@@ -679,7 +693,7 @@ __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, i
                 const int blk = ch / C, c = ch - blk * C;
                 if (blk < sf * sf) {
                     const int dy = blk / sf, dx = blk - dy * sf;
-                    v[k] = (float)rows[((size_t)dy * W + sf * w2 + dx) * c_mem + c];
+                    v[k] = (float)srow[(dy * W + sf * w2 + dx) * c_mem + c];
                 }
             }
         }
@@ -734,11 +748,13 @@ cprune_status regroup_stem_input(const cprune_plan *plan, const void *x, int x_i
     PatchGeometry g;
     if (!patch_geometry(i, &g) || !g.stem || !x || !scratch) return CPRUNE_ERR_INVALID_ARG;
     const unsigned blocks = (unsigned)(i.N * g.He);
+    const size_t row_bytes = (size_t)g.sf * i.W * (x_is_f32 ? (size_t)i.C * 4 : (size_t)i.c_pad * 2);
+    if (row_bytes > 48 * 1024) return CPRUNE_ERR_UNSUPPORTED;     // planning keeps such images off this path
     if (x_is_f32)
-        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3(blocks), dim3(256), 0, st, (const float *)x, i.H, i.W, i.C, i.C, g.sf, g.pad_lo,
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3(blocks), dim3(256), row_bytes, st, (const float *)x, i.H, i.W, i.C, i.C, g.sf, g.pad_lo,
                                          g.WP, (__nv_bfloat162 *)scratch));
     else
-        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16 *)x, i.H, i.W, i.C,
+        CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), row_bytes, st, (const __nv_bfloat16 *)x, i.H, i.W, i.C,
                                          i.c_pad, g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
     return CPRUNE_OK;
 }
