@@ -503,11 +503,26 @@ static double tile_cycles(int MT, int FT, int RS, int cblks, int ksteps_last, in
 // but the MMA's operand reads then cost a full shared-memory cycle per row: measured four times slower.)
 struct PatchGeometry {
     int stem, sf, Re, Se, pad_lo, He, We, WP, cblks, ksteps_last, Wp, kR, kS, pad_w;
+    // the tensors as the kernel addresses them: images x rows x columns of the input (wide tasks) and of the conv output
+    // and the stored output.  A 1x1 stride-1 task is a plain matrix product: its pixels are viewed as ONE row of
+    // N*H*W columns, so that tiles are runs of 128 or 256 pixels with nothing wasted (flat = 1).
+    int flat, vN, vH, vW, vP, vQ, vOH, vOW;
 };
 
 static bool patch_geometry(const cprune_plan_info &i, PatchGeometry *g) {
     if (i.groups != 1) return false;
-    if (i.c_pad >= 16 && i.stride == 1) {
+    g->flat = 0; g->vN = i.N; g->vH = i.H; g->vW = i.W; g->vP = i.P; g->vQ = i.Q; g->vOH = i.out_h; g->vOW = i.out_w;
+    if (i.c_pad >= 16 && i.stride == 1 && i.R == 1 && i.S == 1 && i.pad == 0) {
+        const long long M = (long long)i.N * i.H * i.W;
+        if (M > 0x7fffffffLL) return false;
+        g->flat = 1; g->vN = 1; g->vH = 1; g->vW = (int)M; g->vP = 1; g->vQ = (int)M; g->vOH = 1; g->vOW = (int)M;
+        g->stem = 0; g->sf = 1; g->Re = 1; g->Se = 1; g->pad_lo = 0; g->He = 1; g->We = (int)M; g->WP = (int)M;
+        g->cblks = (i.c_pad + 63) / 64;
+        g->ksteps_last = (i.c_pad - (g->cblks - 1) * 64 + 15) / 16;
+        g->Wp = 128;                           // per tile: set by the planner (128 or 256 pixels)
+        g->kR = 1; g->kS = 1; g->pad_w = 0;
+        return true;
+    } else if (i.c_pad >= 16 && i.stride == 1) {
         if (i.R * i.S <= 1 || i.R > 7 || i.S > 7) return false;
         g->stem = 0; g->sf = 1; g->Re = i.R; g->Se = i.S; g->pad_lo = i.pad; g->He = i.H; g->We = i.W; g->WP = i.W;
         g->cblks = (i.c_pad + 63) / 64;
@@ -552,6 +567,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     if (pool && (plan->opts.residual || (i.P & 1) || (i.Q & 1))) return CPRUNE_ERR_UNSUPPORTED;
     // the 3x3 pool needs tiles narrower than the image, which only tasks without wrap-around slots allow
     if (pool3 && (plan->opts.residual || g.kS != 1)) return CPRUNE_ERR_UNSUPPORTED;
+    if (g.flat && (pool || pool3)) return CPRUNE_ERR_UNSUPPORTED;
     const int k16 = round_up(i.K, 16);
     const int cblks = g.cblks, ksteps_last = g.ksteps_last, RB = 128;
     const int RS = g.kR * g.kS;
@@ -564,8 +580,12 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
       // candidate tile shapes: whole-width rows; for the 3x3 pool (2 tpr + 1) x (2 tpc + 1) conv pixels around tpr x tpc pooled ones
       const int n_shapes = pool3 ? 32 * 32 : 1;
       for (int shape = 0; shape < n_shapes; ++shape) {
-        int TH, TW = i.Q, tiles_w = 1, step_h, step_w = i.Q, org = 0, tiles_per_img, Wp = g.Wp;
-        if (pool3) {
+        int TH, TW = g.vQ, tiles_w = 1, step_h, step_w = g.vQ, org = 0, tiles_per_img, Wp = g.Wp;
+        if (g.flat) {
+            TH = 1; TW = 128 * MT; Wp = TW; step_h = 1; step_w = TW;
+            tiles_w = (g.vQ + TW - 1) / TW;
+            tiles_per_img = tiles_w;
+        } else if (pool3) {
             const int tpr = shape / 32 + 1, tpc = shape % 32 + 1;
             if (tpr > i.out_h || tpc > i.out_w) continue;
             TH = 2 * tpr + 1; TW = 2 * tpc + 1;
@@ -612,7 +632,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
                 if (wstages < 3) continue;
                 if (wstages > 8) wstages = 8;
             }
-            const long long tiles = (long long)i.N * tiles_per_img * tiles_n;
+            const long long tiles = (long long)g.vN * tiles_per_img * tiles_n;
             const double waves = (double)((tiles + 147) / 148);
             double t = waves * tile_cycles(MT, FT, RS, cblks, ksteps_last, RB, Wp, TH, g.kR, resident != 0, acc_bufs);
             if (resident) t += RS * cblks * FT;    // one-time filter load
@@ -625,10 +645,10 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     }
     if (best >= 1e30) return CPRUNE_ERR_UNSUPPORTED;
     // share of accumulator rows that hold real pixels; below one half the im2col kernel is the better choice
-    const double fill = (double)i.P * i.Q / ((double)bt.tiles_per_img * 128 * bt.MT);
+    const double fill = (double)g.vP * g.vQ / ((double)bt.tiles_per_img * 128 * bt.MT);
     if (fill < 0.5) return CPRUNE_ERR_UNSUPPORTED;
     // too few tiles for the SMs: the im2col kernel can split the reduction over more CTAs
-    if ((long long)i.N * bt.tiles_per_img * bt.tiles_n < 64) return CPRUNE_ERR_UNSUPPORTED;
+    if ((long long)g.vN * bt.tiles_per_img * bt.tiles_n < 64) return CPRUNE_ERR_UNSUPPORTED;
     plan->patch = 1;
     plan->pt = bt;
     plan->narrow = g.stem;
@@ -644,7 +664,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     i.tile_n = bt.FT;
     i.tile_k = 64;
     i.stages = bt.wstages;
-    i.tiles_m = i.N * bt.tiles_per_img;
+    i.tiles_m = g.vN * bt.tiles_per_img;
     i.tiles_n = bt.tiles_n;
     i.k_alloc = bt.tiles_n * bt.FT;
     const int ksteps = (cblks - 1) * 4 + ksteps_last;
@@ -787,10 +807,10 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
                 cprune_status s = encode_tiled_bf16_swz(&plan->tm_a, xe, 4, dims, strides, box, 128, true);
                 if (s != CPRUNE_OK) return s;
             } else {
-                const unsigned long long dims[4] = {(unsigned long long)i.c_pad, (unsigned long long)i.W, (unsigned long long)i.H,
-                                                    (unsigned long long)i.N};
-                const unsigned long long strides[3] = {(unsigned long long)i.c_pad * 2, (unsigned long long)i.W * i.c_pad * 2,
-                                                       (unsigned long long)i.H * i.W * i.c_pad * 2};
+                const unsigned long long dims[4] = {(unsigned long long)i.c_pad, (unsigned long long)g.vW, (unsigned long long)g.vH,
+                                                    (unsigned long long)g.vN};
+                const unsigned long long strides[3] = {(unsigned long long)i.c_pad * 2, (unsigned long long)g.vW * i.c_pad * 2,
+                                                       (unsigned long long)g.vH * g.vW * i.c_pad * 2};
                 const unsigned box[4] = {64, (unsigned)Wp, (unsigned)(t.TH + g.kR - 1), 1};
                 cprune_status s = encode_tiled_bf16_swz(&plan->tm_a, xe, 4, dims, strides, box, 128, true);
                 if (s != CPRUNE_OK) return s;
@@ -811,20 +831,20 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
         if (plan->map_y != y) {
             // output [N][P][Q][k_pad]; a store is 64 filters x Wp pixels x TH rows (see the epilogue).  With a fused
             // pool the kernel stores by hand and the map is not used.
-            const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)i.out_w, (unsigned long long)i.out_h,
-                                                (unsigned long long)i.N};
-            const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)i.out_w * i.k_pad * 2,
-                                                   (unsigned long long)i.out_h * i.out_w * i.k_pad * 2};
+            const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)g.vOW, (unsigned long long)g.vOH,
+                                                (unsigned long long)g.vN};
+            const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)g.vOW * i.k_pad * 2,
+                                                   (unsigned long long)g.vOH * g.vOW * i.k_pad * 2};
             const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
             cprune_status s = encode_tiled_bf16_swz(&plan->tm_y, y, 4, dims, strides, box, 128, false);
             if (s != CPRUNE_OK) return s;
             plan->map_y = y;
         }
         if (res && plan->map_res != res) {
-            const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)i.Q, (unsigned long long)i.P,
-                                                (unsigned long long)i.N};
-            const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)i.Q * i.k_pad * 2,
-                                                   (unsigned long long)i.P * i.Q * i.k_pad * 2};
+            const unsigned long long dims[4] = {(unsigned long long)i.k_pad, (unsigned long long)g.vQ, (unsigned long long)g.vP,
+                                                (unsigned long long)g.vN};
+            const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)g.vQ * i.k_pad * 2,
+                                                   (unsigned long long)g.vP * g.vQ * i.k_pad * 2};
             const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
             cprune_status s = encode_tiled_bf16_swz(&plan->tm_res, res, 4, dims, strides, box, 128, true);
             if (s != CPRUNE_OK) return s;
@@ -845,9 +865,9 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
         }
     }
     PatchParams p;
-    p.P = i.P; p.Q = i.Q; p.Wp = Wp; p.TH = t.TH; p.tiles_per_img = t.tiles_per_img;
+    p.P = g.vP; p.Q = g.vQ; p.Wp = Wp; p.TH = t.TH; p.tiles_per_img = t.tiles_per_img;
     p.TW = t.TW; p.tiles_w = t.tiles_w; p.step_h = t.step_h; p.step_w = t.step_w; p.org = t.org;
-    p.out_h = i.out_h; p.out_w = i.out_w;
+    p.out_h = g.vOH; p.out_w = g.vOW;
     p.tiles_m = i.tiles_m; p.tiles_n = i.tiles_n; p.FT = t.FT; p.MT = t.MT; p.R = g.kR; p.S = g.kS; p.pad = g.pad_lo; p.pad_w = g.pad_w;
     p.cblks = g.cblks;
     p.ksteps_last = g.ksteps_last;
