@@ -170,6 +170,16 @@ def test_fused_maxpool(cp, case):
     check_task(cp, N, C, HW, HW, K, 3, 1, 1, act="relu", pool="max2x2", kernel="tensor")
 
 
+def test_pointwise_tasks_as_flat_matrix_products(cp):
+    # 1x1 stride-1 tasks with enough pixels run on the patch kernel with all pixels viewed as one row: ragged last tile,
+    # residual through the staging buffer, several filter tiles, channel counts off the 16 / 64 grid
+    plan = check_task(cp, 8, 24, 56, 56, 108, 1, 1, 0, act="relu6", kernel="tensor")
+    assert plan.variant == 1
+    check_task(cp, 3, 108, 57, 59, 24, 1, 1, 0, act="none", with_res=True, kernel="tensor")
+    check_task(cp, 5, 72, 40, 41, 300, 1, 1, 0, act="relu", kernel="tensor")
+    check_task(cp, 64, 320, 7, 7, 1280, 1, 1, 0, act="relu6", kernel="tensor")
+
+
 def test_stems_on_the_patch_kernel(cp):
     # enough tiles for the patch kernel: the input is regrouped into 16-channel pixels (stride 1 and 2)
     plan = check_task(cp, 16, 3, 64, 64, 64, 7, 2, 3, kernel="tensor")
