@@ -64,6 +64,12 @@ struct PatchParams {
     int *status;
 };
 
+// Maximum of 8 non-negative bf16 values (after ReLU / ReLU6; max.f32 never yields -0): their bit patterns order like
+// unsigned integers, so one SIMD integer instruction handles two values.
+__device__ __forceinline__ uint4 bf16x8_max_nonneg(uint4 a, uint4 b) {
+    return make_uint4(__vmaxu2(a.x, b.x), __vmaxu2(a.y, b.y), __vmaxu2(a.z, b.z), __vmaxu2(a.w, b.w));
+}
+
 __device__ __forceinline__ uint4 bf16x8_max(uint4 a, uint4 b) {
     uint4 r;
     __nv_bfloat162 *pa = reinterpret_cast<__nv_bfloat162 *>(&a), *pb = reinterpret_cast<__nv_bfloat162 *>(&b);
@@ -295,9 +301,28 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         };
         // activation as a clamp: no branches in the per-element code
         const float act_lo = p.act == CPRUNE_ACT_NONE ? -INFINITY : 0.f, act_hi = p.act == CPRUNE_ACT_RELU6 ? 6.f : INFINITY;
+        const bool clamp_lo = p.act != CPRUNE_ACT_NONE;      // results are >= 0
         const bool store_thread = warp == PK_FIRST_EPI && lane == 0;
         const int groups = (p.FT + 63) / 64;
         const int n_entries = p.pool == 1 ? (p.TH >> 1) * (p.Q >> 1) : ((p.TH - 1) >> 1) * ((p.TW - 1) >> 1);
+        // 3x3 pool: a thread copies out at most two (pooled pixel, 8 filters) items per tile, the same ones in every tile;
+        // the shared-memory offsets of their nine window slots are worked out once
+        uint32_t win_off[2][9];
+        int win_pi[2] = {0, 0}, win_pj[2] = {0, 0};
+        if (p.pool == 2) {
+            const int tpc = (p.TW - 1) >> 1;
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+                const int e = etid + it * 256;
+                const int ent = e >> 3, chunk = e & 7;
+                win_pi[it] = ent / tpc; win_pj[it] = ent - win_pi[it] * tpc;
+#pragma unroll
+                for (int k = 0; k < 9; ++k) {
+                    const int sl = (2 * win_pi[it] + k / 3) * p.Wp + 2 * win_pj[it] + k % 3;
+                    win_off[it][k] = (uint32_t)((sl >> 7) * PK_BLOCK_BYTES) + sub_off(sl & 127, chunk);
+                }
+            }
+        }
         // The residual of a group arrives by TMA in the staging buffer the group will use (same box as the store:
         // wrap-around slots read as zero); the values are added there in place.  The load for the next group is
         // issued as soon as its buffer is free.
@@ -427,28 +452,38 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     // windows of (TH - 1) / 2 x (TW - 1) / 2 pooled pixels.  All nine slots of a window are inside the
                     // staged tile, so they are loaded unconditionally; conv pixels outside the image are replaced by
                     // -inf (they never win).
-                    const int tpc = (p.TW - 1) >> 1;
                     const int pr0 = (p0 + 1) >> 1, pc0 = (q0 + 1) >> 1;
                     const uint4 ninf = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-                    for (int e = etid; e < n_entries * 8; e += 256) {
-                        const int ent = e >> 3, chunk = e & 7;
-                        const int pi = ent / tpc, pj = ent - pi * tpc;
-                        const int pr = pr0 + pi, pc = pc0 + pj;
-                        if (pr < p.out_h && pc < p.out_w && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
-                            const int r0 = p0 + 2 * pi, c0 = q0 + 2 * pj, s0 = 2 * pi * p.Wp + 2 * pj;
+                    // after ReLU / ReLU6 all values are >= 0: pixels outside the image can be replaced by 0 (every
+                    // window holds a real pixel) and the maximum taken on the bit patterns
+                    const uint4 fill = clamp_lo ? make_uint4(0u, 0u, 0u, 0u) : ninf;
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int e = etid + it * 256;
+                        const int chunk = e & 7;
+                        const int pr = pr0 + win_pi[it], pc = pc0 + win_pj[it];
+                        if (e < n_entries * 8 && pr < p.out_h && pc < p.out_w && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
+                            const int r0 = p0 + 2 * win_pi[it], c0 = q0 + 2 * win_pj[it];
+                            // bit d of a mask: window row / column d lies inside the image
+                            const uint32_t rmask = (r0 >= 0 ? 1u : 0u) | 2u | (r0 + 2 < p.P ? 4u : 0u);
+                            const uint32_t cmask = (c0 >= 0 ? 1u : 0u) | 2u | (c0 + 2 < p.Q ? 4u : 0u);
                             uint4 w[9];
 #pragma unroll
-                            for (int di = 0; di < 3; ++di)
-#pragma unroll
-                                for (int dj = 0; dj < 3; ++dj) {
-                                    const bool inside = r0 + di >= 0 && r0 + di < p.P && c0 + dj >= 0 && c0 + dj < p.Q;
-                                    const uint4 t = staged(s0 + di * p.Wp + dj, chunk);
-                                    w[di * 3 + dj] = inside ? t : ninf;
-                                }
-                            const uint4 a0 = bf16x8_max(bf16x8_max(w[0], w[1]), bf16x8_max(w[2], w[3]));
-                            const uint4 a1 = bf16x8_max(bf16x8_max(w[4], w[5]), bf16x8_max(w[6], w[7]));
-                            *(uint4 *)(p.y + (((size_t)n * p.out_h + pr) * p.out_w + pc) * p.k_pad + kg + chunk * 8) =
-                                bf16x8_max(bf16x8_max(a0, a1), w[8]);
+                            for (int k = 0; k < 9; ++k) {
+                                const uint4 t = *(const uint4 *)(buf + win_off[it][k]);
+                                w[k] = ((rmask >> (k / 3)) & (cmask >> (k % 3)) & 1u) ? t : fill;
+                            }
+                            uint4 m;
+                            if (clamp_lo) {
+                                const uint4 a0 = bf16x8_max_nonneg(bf16x8_max_nonneg(w[0], w[1]), bf16x8_max_nonneg(w[2], w[3]));
+                                const uint4 a1 = bf16x8_max_nonneg(bf16x8_max_nonneg(w[4], w[5]), bf16x8_max_nonneg(w[6], w[7]));
+                                m = bf16x8_max_nonneg(bf16x8_max_nonneg(a0, a1), w[8]);
+                            } else {
+                                const uint4 a0 = bf16x8_max(bf16x8_max(w[0], w[1]), bf16x8_max(w[2], w[3]));
+                                const uint4 a1 = bf16x8_max(bf16x8_max(w[4], w[5]), bf16x8_max(w[6], w[7]));
+                                m = bf16x8_max(bf16x8_max(a0, a1), w[8]);
+                            }
+                            *(uint4 *)(p.y + (((size_t)n * p.out_h + pr) * p.out_w + pc) * p.k_pad + kg + chunk * 8) = m;
                         }
                     }
                 }
