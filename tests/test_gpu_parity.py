@@ -201,6 +201,49 @@ def test_maxpool_3x3_stride_2(cp, case):
     assert plan.out_h == (P - 1) // 2 + 1
 
 
+@pytest.mark.parametrize("case", [
+    # tasks of the benchmarked models at their full batch-64 sizes, i.e. in the launch configuration bench.py times:
+    # N, C, H, W, K, R, stride, pad, groups, act, residual, pool
+    (64, 3, 224, 224, 64, 7, 2, 3, 1, "relu", False, "max3x3s2"),      # ResNet stem with its pool (patch kernel, regrouped)
+    (64, 64, 56, 56, 44, 3, 1, 1, 1, "relu", False, None),             # stage 1 conv1 (patch kernel, resident filters)
+    (64, 179, 14, 14, 256, 3, 1, 1, 1, "relu", True, None),            # stage 3 conv2 + residual (patch kernel, streamed)
+    (64, 512, 7, 7, 358, 3, 1, 1, 1, "relu", False, None),             # stage 4 (im2col kernel)
+    (64, 64, 56, 56, 89, 3, 2, 1, 1, "relu", False, None),             # stride-2 3x3 (im2col kernel)
+    (64, 16, 112, 112, 72, 1, 1, 0, 1, "relu6", False, None),          # MobileNetV2 expand (flat matrix product)
+    (64, 72, 112, 112, 72, 3, 2, 1, 72, "relu6", False, None)])        # depthwise, stride 2
+def test_full_size_tasks_on_sampled_outputs(cp, case):
+    N, C, H, W, K, R, stride, pad, groups, act, with_res, pool = case
+    P, Q = oracle.out_size(H, R, stride, pad), oracle.out_size(W, R, stride, pad)
+    x, w, b, res = wl.conv_task_tensors(31, N, C, H, W, K, R, R, groups, with_res, P, Q)
+    y, plan = run_task(cp, x, w, b, stride, pad, groups, act, res, pool)
+    rng = np.random.default_rng(5)
+    n_pts = 192
+    oh, ow = plan.out_h, plan.out_w
+    pts = np.stack([rng.integers(0, N, n_pts), rng.integers(0, oh, n_pts), rng.integers(0, ow, n_pts),
+                    rng.integers(0, K, n_pts)], axis=1)
+    # corners and edges are where padding, ragged tiles and pooling windows go wrong
+    pts[:8, 1:3] = [[0, 0], [0, ow - 1], [oh - 1, 0], [oh - 1, ow - 1], [0, ow // 2], [oh // 2, 0], [oh - 1, ow // 2], [oh // 2, ow - 1]]
+    pts[:4, 0] = [0, N - 1, 0, N - 1]
+    if pool is None:
+        ref, bound = oracle.conv2d_points(x, w, b, stride, pad, groups, act, res, pts)
+    else:
+        ref = np.full(n_pts, -np.inf)
+        bound = np.zeros(n_pts)
+        for di in range(3):
+            for dj in range(3):
+                q = pts.copy()
+                q[:, 1] = 2 * pts[:, 1] - 1 + di
+                q[:, 2] = 2 * pts[:, 2] - 1 + dj
+                inside = (q[:, 1] >= 0) & (q[:, 1] < P) & (q[:, 2] >= 0) & (q[:, 2] < Q)
+                v, bd = oracle.conv2d_points(x, w, b, stride, pad, groups, act, res, q[inside])
+                ref[inside] = np.maximum(ref[inside], v)
+                bound[inside] = np.maximum(bound[inside], bd)
+    got = y[pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3]]
+    worst = np.max(np.abs(got - ref) / (bound + 1e-30))
+    assert worst <= TOL, (worst, pts[np.argmax(np.abs(got - ref) / (bound + 1e-30))])
+    assert np.all(y[..., K:] == 0)
+
+
 @pytest.mark.parametrize("C", [64, 65, 66, 67, 68, 69, 70, 71, 72, 73, 79, 80, 81])
 def test_every_channel_residue(cp, C):
     # C and K sweep the residues modulo 8 and 16 around a 64-channel block boundary
