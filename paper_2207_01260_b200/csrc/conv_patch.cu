@@ -103,6 +103,30 @@ __device__ __forceinline__ void issue_tap(uint32_t d_tmem, uint32_t a_lo, uint32
     __syncwarp();
 }
 
+// A whole filter row (S taps) from one elected block: used when nothing has to be waited for between taps.
+__device__ __forceinline__ void issue_row(uint32_t d_tmem, uint32_t a_lo, uint32_t w_lo, uint32_t desc_hi, uint32_t idesc,
+                                          uint32_t accumulate, int nk, int S, uint32_t slot_step, uint32_t w_step, uint32_t commit_p) {
+    if (elect_one()) {
+        for (int s = 0; s < S; ++s) {
+            if (nk == 4) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_words(d_tmem, a_lo + (uint32_t)(2 * kk), w_lo + (uint32_t)(2 * kk), desc_hi, idesc, kk ? 1u : accumulate);
+            } else {
+                umma_bf16_words(d_tmem, a_lo, w_lo, desc_hi, idesc, accumulate);
+#pragma unroll
+                for (int kk = 1; kk < 3; ++kk)
+                    if (kk < nk) umma_bf16_words(d_tmem, a_lo + (uint32_t)(2 * kk), w_lo + (uint32_t)(2 * kk), desc_hi, idesc, 1u);
+            }
+            accumulate = 1;
+            a_lo += slot_step;
+            w_lo += w_step;
+        }
+        if (commit_p) umma_commit(commit_p);
+    }
+    __syncwarp();
+}
+
 // First output pixel (may be -1 with the 3x3 pool, whose windows reach one pixel outside the tile's own pooled
 // pixels) and image of tile tm.
 __device__ __forceinline__ void tile_origin(const PatchParams &p, int tm, int &n, int &p0, int &q0) {
@@ -259,20 +283,31 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (!ok) break;
                 const int nk = cb == p.cblks - 1 ? p.ksteps_last : 4;
                 uint32_t tap_lo = patch_lo + (uint32_t)(mb * 128) * slot_step;      // the second block's slots follow the first's
-                int s = 0;
-                for (int tap = 0; tap < RS; ++tap) {
-                    // resident filters: the barrier completes once (first tile) and stays complete for parity 0
-                    ok = __all_sync(0xffffffffu, mbar_wait(wfull(ws), p.resident ? 0u : wphase, abort_flag, p.status));
-                    if (!ok) break;
-                    {
-                        const uint32_t cw = p.resident ? 0u : wempty(ws), cp = tap == RS - 1 ? pempty(ps) : 0u;
-                        issue_tap(d_tmem, tap_lo, w_lo, desc_hi, idesc, accumulate, nk, cw, cp);
+                if (p.resident && item != (int)blockIdx.x) {
+                    // resident filters, loaded during the first tile: nothing to wait for, a filter row per elected block
+                    for (int r = 0; r < p.R; ++r) {
+                        issue_row(d_tmem, tap_lo, w_lo, desc_hi, idesc, accumulate, nk, p.S, slot_step, w_step, r == p.R - 1 ? pempty(ps) : 0u);
+                        accumulate = 1;
+                        tap_lo += (uint32_t)p.Wp * slot_step;
+                        w_lo += (uint32_t)p.S * w_step;
+                        ws += p.S;
+                        if (ws == p.wstages) { ws = 0; w_lo = w_lo0; }
                     }
-                    accumulate = 1;
-                    w_lo += w_step;
-                    if (++ws == p.wstages) { ws = 0; wphase ^= 1u; w_lo = w_lo0; }
-                    tap_lo += slot_step;
-                    if (++s == p.S) { s = 0; tap_lo += row_step - slot_step; }
+                } else {
+                    int s = 0;
+                    for (int tap = 0; tap < RS; ++tap) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(wfull(ws), p.resident ? 0u : wphase, abort_flag, p.status));
+                        if (!ok) break;
+                        {
+                            const uint32_t cw = p.resident ? 0u : wempty(ws), cp = tap == RS - 1 ? pempty(ps) : 0u;
+                            issue_tap(d_tmem, tap_lo, w_lo, desc_hi, idesc, accumulate, nk, cw, cp);
+                        }
+                        accumulate = 1;
+                        w_lo += w_step;
+                        if (++ws == p.wstages) { ws = 0; wphase ^= 1u; w_lo = w_lo0; }
+                        tap_lo += slot_step;
+                        if (++s == p.S) { s = 0; tap_lo += row_step - slot_step; }
+                    }
                 }
                 patch_lo += patch_step;
                 if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; patch_lo = patch_lo0; }
