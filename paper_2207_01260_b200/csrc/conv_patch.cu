@@ -688,8 +688,12 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             const int w_stage = round_up(FT * RB, 1024);
             int staging_bufs = sb_max, wstages = 0, resident = 0;
             // resident filters when the whole set of this filter tile fits
-            if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES) {
-                for (int sb = sb_max; sb >= sb_min && !resident; --sb)
+            // (with a residual, only beside two staging buffers: with one buffer the residual of a group can only be
+            // fetched after the previous group's store has drained, which costs more than streaming the filters)
+            const char *force_res = getenv("CPRUNE_PATCH_RESIDENT");      // measurement override: 0 = never, 1 = whenever it fits
+            const int sb_res_min = (plan->opts.residual && !(force_res && force_res[0] == '1')) ? 2 : sb_min;
+            if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES && !(force_res && force_res[0] == '0')) {
+                for (int sb = sb_max; sb >= sb_res_min && !resident; --sb)
                     if (RS * cblks * w_stage + sb * MT * PK_BLOCK_BYTES <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
             }
             if (!resident) {
