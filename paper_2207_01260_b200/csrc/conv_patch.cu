@@ -44,7 +44,7 @@ constexpr int PK_MMA_WARP = 3;
 constexpr int PK_FIRST_EPI = 4;
 constexpr int PK_MMA_WARP2 = 12;         // issues for the second accumulator block when MT = 2
 constexpr int PK_MAX_WSTAGES = 32;
-constexpr int PK_PATCH_STAGES = 2;
+constexpr int PK_MAX_PATCH_STAGES = 4;   // patch ring: 2 stages, more for tasks with small patches and several channel blocks
 constexpr int PK_CTRL_BYTES = 3072;      // barriers (1 KB) + slot table (2 KB)
 constexpr int PK_BLOCK_BYTES = 16384;    // staged block: 128 slots x 64 filters bf16
 
@@ -53,7 +53,7 @@ struct PatchParams {
     int TW, tiles_w, step_h, step_w, org;   // tile (ty, tx) starts at output (ty * step_h + org, tx * step_w + org) and spans TH x TW
     int out_h, out_w;                       // stored extent (after a fused pool)
     int FT, MT, R, S, pad, pad_w, cblks, ksteps_last, k_pad;   // pad: rows above the image in a patch; pad_w: columns left of it
-    int act, wstages, resident, acc_bufs, staging_bufs, pool;
+    int act, wstages, pstages, resident, acc_bufs, staging_bufs, pool;
     int patch_bytes;       // shared memory of one patch stage
     int patch_box_bytes;   // bytes one patch load delivers
     int w_stage_bytes;     // shared memory of one filter stage (FT rows, rounded up to 1024 bytes)
@@ -149,19 +149,19 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const uint32_t w_bytes = (uint32_t)p.w_stage_bytes;                   // stage stride
     const uint32_t w_tx_bytes = (uint32_t)p.FT * 16u * (uint32_t)p.rb16;  // bytes one filter load delivers
     const uint32_t patch0 = base;
-    const uint32_t w0 = patch0 + PK_PATCH_STAGES * (uint32_t)p.patch_bytes;
+    const uint32_t w0 = patch0 + (uint32_t)p.pstages * (uint32_t)p.patch_bytes;
     const uint32_t staging0 = w0 + (uint32_t)p.wstages * w_bytes;
     const uint32_t stage_buf_bytes = (uint32_t)p.MT * PK_BLOCK_BYTES;
     const uint32_t ctrl0 = staging0 + (uint32_t)p.staging_bufs * stage_buf_bytes;
     uint8_t *ctrl = smem + (ctrl0 - base);
     auto pfull = [&](int s) { return ctrl0 + 8u * s; };
-    auto pempty = [&](int s) { return ctrl0 + 16u + 8u * s; };
-    auto tfull = [&](int a) { return ctrl0 + 32u + 8u * a; };
-    auto tempty = [&](int a) { return ctrl0 + 48u + 8u * a; };
-    const uint32_t epi_bar = ctrl0 + 64u;
-    auto res_full = [&](int b) { return ctrl0 + 80u + 8u * b; };   // residual tile landed in staging buffer b
-    uint32_t *tmem_slot = (uint32_t *)(ctrl + 72);
-    volatile int *abort_flag = (volatile int *)(ctrl + 76);
+    auto pempty = [&](int s) { return ctrl0 + 32u + 8u * s; };
+    auto tfull = [&](int a) { return ctrl0 + 64u + 8u * a; };
+    auto tempty = [&](int a) { return ctrl0 + 80u + 8u * a; };
+    const uint32_t epi_bar = ctrl0 + 96u;
+    auto res_full = [&](int b) { return ctrl0 + 112u + 8u * b; };   // residual tile landed in staging buffer b
+    uint32_t *tmem_slot = (uint32_t *)(ctrl + 104);
+    volatile int *abort_flag = (volatile int *)(ctrl + 108);
     auto wfull = [&](int s) { return ctrl0 + 128u + 8u * s; };
     auto wempty = [&](int s) { return ctrl0 + 384u + 8u * s; };
     int2 *lut = (int2 *)(ctrl + 1024);   // entry -> (source slot | tile row << 16, output offset in elements); x < 0: nothing to store
@@ -173,7 +173,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 
     if (threadIdx.x == 0) {
         // every accumulator block has its own issuing warp: stages are free, and a tile is complete, once all have committed
-        for (int s = 0; s < PK_PATCH_STAGES; ++s) { mbar_init(pfull(s), 1); mbar_init(pempty(s), p.MT); }
+        for (int s = 0; s < p.pstages; ++s) { mbar_init(pfull(s), 1); mbar_init(pempty(s), p.MT); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull(a), p.MT); mbar_init(tempty(a), 8); }
         for (int s = 0; s < p.wstages; ++s) { mbar_init(wfull(s), 1); mbar_init(wempty(s), p.MT); }
         mbar_init(epi_bar, 8);
@@ -183,9 +183,9 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // slot table: which accumulator rows hold real output pixels and where they go
-    for (int e = threadIdx.x; e < 256; e += PK_THREADS) {
+    for (int e = threadIdx.x; e < 256 && p.pool == 1; e += PK_THREADS) {
         int2 v = make_int2(-1, 0);
-        if (p.pool == 1) {
+        {
             const int hq = p.Q >> 1;
             const int i2 = e / hq, j2 = e - i2 * hq;
             if (i2 < (p.TH >> 1)) v = make_int2((2 * i2 * p.Wp + 2 * j2) | ((2 * i2) << 16), (i2 * hq + j2) * p.k_pad);
@@ -222,7 +222,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     tma_load_4d(patch0 + (uint32_t)ps * p.patch_bytes, &tm_x, pfull(ps), cb * 64, q0 - p.pad_w, p0 - p.pad, n);
                 }
                 __syncwarp();
-                if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; }
+                if (++ps == p.pstages) { ps = 0; pphase ^= 1u; }
             }
         }
     } else if (warp < PK_MMA_WARP) {
@@ -310,7 +310,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     }
                 }
                 patch_lo += patch_step;
-                if (++ps == PK_PATCH_STAGES) { ps = 0; pphase ^= 1u; patch_lo = patch_lo0; }
+                if (++ps == p.pstages) { ps = 0; pphase ^= 1u; patch_lo = patch_lo0; }
             }
             if (ok && elect_one()) umma_commit(tfull(acc));
             __syncwarp();
@@ -682,7 +682,11 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             const int acc_bufs = 2 * MT * FT <= 512 ? 2 : 1;
             const int patch_bytes = round_up((128 * MT + (g.kR - 1) * Wp + g.kS - 1) * RB, 1024);
             if (patch_bytes < Wp * (TH + g.kR - 1) * RB) continue;
-            const int fixed = 1024 + PK_PATCH_STAGES * patch_bytes + PK_CTRL_BYTES;
+            // patch ring depth: two stages; up to four when the task has that many channel blocks and the patches are
+            // small (1x1 tasks), because each load's latency is otherwise exposed
+            int pstages = 2;
+            if (cblks > 2 && patch_bytes <= 32 * 1024) pstages = cblks < PK_MAX_PATCH_STAGES ? cblks : PK_MAX_PATCH_STAGES;
+            const int fixed = 1024 + pstages * patch_bytes + PK_CTRL_BYTES;
             const int budget = 227 * 1024 - fixed;
             const int sb_max = 2, sb_min = 1;
             const int w_stage = round_up(FT * RB, 1024);
@@ -712,7 +716,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             if (resident) t += RS * cblks * FT;    // one-time filter load
             if (t < best) {
                 best = t;
-                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org};
+                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org, pstages};
             }
         }
       }
@@ -743,7 +747,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     i.k_alloc = bt.tiles_n * bt.FT;
     const int ksteps = (cblks - 1) * 4 + ksteps_last;
     i.padded_flops = 2.0 * (double)i.tiles_m * i.tile_m * (double)i.k_alloc * RS * ksteps * 16.0;
-    plan->smem_bytes = 1024 + PK_PATCH_STAGES * bt.patch_bytes + bt.wstages * round_up(bt.FT * RB, 1024) +
+    plan->smem_bytes = 1024 + bt.pstages * bt.patch_bytes + bt.wstages * round_up(bt.FT * RB, 1024) +
                        bt.staging_bufs * bt.MT * PK_BLOCK_BYTES + PK_CTRL_BYTES;
     return CPRUNE_OK;
 }
@@ -947,7 +951,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     p.ksteps_last = g.ksteps_last;
     p.k_pad = i.k_pad;
     p.act = plan->opts.activation;
-    p.wstages = t.wstages; p.resident = t.resident; p.acc_bufs = t.acc_bufs; p.staging_bufs = t.staging_bufs;
+    p.wstages = t.wstages; p.pstages = t.pstages; p.resident = t.resident; p.acc_bufs = t.acc_bufs; p.staging_bufs = t.staging_bufs;
     p.pool = plan->fused_pool ? plan->opts.pool : 0;
     p.patch_bytes = t.patch_bytes;
     p.patch_box_bytes = Wp * (t.TH + g.kR - 1) * 128;

@@ -14,6 +14,7 @@
 struct PatchTiling {
     int MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes;
     int TW, tiles_w, step_h, step_w, org;   // tile width, tiles per image row, distance between tiles, origin offset
+    int pstages;                            // depth of the patch ring
 };
 
 struct cprune_plan {
