@@ -77,10 +77,9 @@ __global__ void __launch_bounds__(256) gap_kernel(const bf16x8 *__restrict__ x, 
     }
 }
 
-// one warp per (output feature o, group of NB images): the warp reads the weight row once and
-// NB activation rows, reduces with shuffles; warps of a block share o when there are enough groups,
-// so the weight row is fetched from L2 once per block
-template <int NB>
+// One warp per (OB consecutive output features, group of NB images): the lanes split the input features; every
+// activation chunk is used for OB outputs and every weight chunk for NB images, reduced with shuffles at the end.
+template <int NB, int OB>
 __global__ void __launch_bounds__(256) fc_kernel(const bf16x8 *__restrict__ x, int N, int in8,
                                                  const bf16x8 *__restrict__ w, const float *__restrict__ b, int out,
                                                  int out_pad, int act, int out_is_f32, void *__restrict__ y) {
@@ -89,36 +88,44 @@ __global__ void __launch_bounds__(256) fc_kernel(const bf16x8 *__restrict__ x, i
     const int ngroups = (N + NB - 1) / NB;
     const long long widx = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (widx >= (long long)out_pad * ngroups) return;
-    const int o = (int)(widx / ngroups);
-    const int n0 = (int)(widx - (long long)o * ngroups) * NB;
-    const bf16x8 *wr = w + (size_t)o * in8;
-    float acc[NB];
+    if (widx >= (long long)(out_pad / OB) * ngroups) return;
+    const int o0 = (int)(widx / ngroups) * OB;
+    const int n0 = (int)(widx % ngroups) * NB;
+    float acc[OB][NB];
 #pragma unroll
-    for (int j = 0; j < NB; ++j) acc[j] = 0.f;
+    for (int q = 0; q < OB; ++q)
+#pragma unroll
+        for (int j = 0; j < NB; ++j) acc[q][j] = 0.f;
     for (int i = lane; i < in8; i += 32) {
-        float wf[8];
-        unpack8(ldg8(wr + i), wf);
+        float wf[OB][8];
+#pragma unroll
+        for (int q = 0; q < OB; ++q) unpack8(ldg8(w + (size_t)(o0 + q) * in8 + i), wf[q]);
 #pragma unroll
         for (int j = 0; j < NB; ++j) {
             if (n0 + j < N) {
                 float xf[8];
                 unpack8(ldg8(x + (size_t)(n0 + j) * in8 + i), xf);
 #pragma unroll
-                for (int t = 0; t < 8; ++t) acc[j] = fmaf(xf[t], wf[t], acc[j]);
+                for (int q = 0; q < OB; ++q)
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) acc[q][j] = fmaf(xf[t], wf[q][t], acc[q][j]);
             }
         }
     }
 #pragma unroll
-    for (int j = 0; j < NB; ++j) {
-        float v = acc[j];
-        for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-        if (lane == 0 && n0 + j < N) {
-            v = apply_act(v + b[o], act);
-            if (out_is_f32) {
-                if (o < out) ((float *)y)[(size_t)(n0 + j) * out + o] = v;
-            } else {
-                ((__nv_bfloat16 *)y)[(size_t)(n0 + j) * out_pad + o] = __float2bfloat16_rn(o < out ? v : 0.f);
+    for (int q = 0; q < OB; ++q) {
+        const int o = o0 + q;
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            float v = acc[q][j];
+            for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+            if (lane == 0 && n0 + j < N) {
+                v = apply_act(v + b[o], act);
+                if (out_is_f32) {
+                    if (o < out) ((float *)y)[(size_t)(n0 + j) * out + o] = v;
+                } else {
+                    ((__nv_bfloat16 *)y)[(size_t)(n0 + j) * out_pad + o] = __float2bfloat16_rn(o < out ? v : 0.f);
+                }
             }
         }
     }
@@ -163,8 +170,8 @@ cprune_status cprune_fc(const void *x, int N, int in, const void *w_packed, cons
     if (!x || !w_packed || !b_packed || !y || N <= 0 || in <= 0 || out <= 0) return CPRUNE_ERR_INVALID_ARG;
     int in8 = cprune_padded_channels(in) / 8, out_pad = cprune_padded_channels(out);
     const int warps = 8;
-    const long long total_warps = (long long)out_pad * ((N + 7) / 8);
-    CPRUNE_CUDA_CHECK(launch_chained(fc_kernel<8>, dim3((unsigned)((total_warps + warps - 1) / warps)), dim3(warps * 32), 0, (cudaStream_t)stream,
+    const long long total_warps = (long long)(out_pad / 4) * ((N + 7) / 8);
+    CPRUNE_CUDA_CHECK(launch_chained(fc_kernel<8, 4>, dim3((unsigned)((total_warps + warps - 1) / warps)), dim3(warps * 32), 0, (cudaStream_t)stream,
                                      (const bf16x8 *)x, N, in8, (const bf16x8 *)w_packed, b_packed, out, out_pad, act, out_is_f32, y));
     return CPRUNE_OK;
 }
