@@ -171,15 +171,14 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int RS = p.R * p.S;
 
-    if (threadIdx.x == 0) {
-        // every accumulator block has its own issuing warp: stages are free, and a tile is complete, once all have committed
-        for (int s = 0; s < p.pstages; ++s) { mbar_init(pfull(s), 1); mbar_init(pempty(s), p.MT); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull(a), p.MT); mbar_init(tempty(a), 8); }
-        for (int s = 0; s < p.wstages; ++s) { mbar_init(wfull(s), 1); mbar_init(wempty(s), p.MT); }
-        mbar_init(epi_bar, 8);
-        mbar_init(res_full(0), 1);
-        mbar_init(res_full(1), 1);
-        *abort_flag = 0;
+    // barrier set-up, spread over the lanes of warp 0 (one thread doing up to 70 initialisations costs microseconds).
+    // Every accumulator block has its own issuing warp: stages are free, and a tile is complete, once all have committed.
+    if (threadIdx.x < 32) {
+        const int l = threadIdx.x;
+        if (l < p.pstages) { mbar_init(pfull(l), 1); mbar_init(pempty(l), p.MT); }
+        if (l < 2) { mbar_init(tfull(l), p.MT); mbar_init(tempty(l), 8); mbar_init(res_full(l), 1); }
+        if (l == 2) { mbar_init(epi_bar, 8); *abort_flag = 0; }
+        if (l < p.wstages) { mbar_init(wfull(l), 1); mbar_init(wempty(l), p.MT); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // slot table: which accumulator rows hold real output pixels and where they go
