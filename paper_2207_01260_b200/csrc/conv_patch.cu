@@ -602,7 +602,7 @@ static bool patch_geometry(const cprune_plan_info &i, PatchGeometry *g) {
     } else if (i.c_pad == 8 && i.stride <= 2 && i.C * i.stride * i.stride <= 16 && i.R * i.S > 1 && i.R <= 8 && i.S <= 8) {
         const int sf = i.stride;
         if ((i.H % sf) || (i.W % sf)) return false;
-        if ((size_t)sf * i.W * 16 > 48 * 1024) return false;      // the regrouping pass stages sf input rows in shared memory
+        if ((size_t)4 * sf * i.W * 16 > 48 * 1024) return false;   // the regrouping pass stages 4 * sf input rows in shared memory
         if (i.R - 1 - i.pad < 0 || i.S - 1 - i.pad < 0) return false;
         g->stem = 1; g->sf = sf;
         g->pad_lo = sf == 1 ? i.pad : (i.pad + 1) / 2;
@@ -756,20 +756,32 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
 // whatever follows the image) are zero:
 //   out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
 // Eight threads per output pixel, two channels each: the 32 bytes of a pixel are written by neighbouring lanes.
+constexpr int RG_ROWS = 4;     // regrouped rows per block
+
 template <typename T>
 __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, int H, int W, int C, int c_mem, int sf, int pad_lo, int WP,
                                                       __nv_bfloat162 *__restrict__ out) {
     pdl_trigger();
     pdl_wait();
-    // one block per output row (image n, regrouped row h2): its sf input rows are contiguous in memory and are
+    // one block per RG_ROWS regrouped rows of one image: their sf * RG_ROWS input rows are contiguous in memory and are
     // brought into shared memory with 16-byte loads first
     extern __shared__ __align__(16) unsigned char rg_smem[];
+    __shared__ int src_off[16];            // regrouped channel -> offset within an sf x sf input block, or -1 (zero)
     T *srow = reinterpret_cast<T *>(rg_smem);
     const int H2 = H / sf, W2 = W / sf;
-    const int n = blockIdx.x / H2, h2 = blockIdx.x - n * H2;
-    const T *rows = x + ((size_t)n * H + (size_t)sf * h2) * W * c_mem;
-    const int n_elems = sf * W * c_mem;
+    const int blocks_per_img = (H2 + RG_ROWS - 1) / RG_ROWS;
+    const int n = blockIdx.x / blocks_per_img;
+    const int h2_0 = (blockIdx.x - n * blocks_per_img) * RG_ROWS;
+    const int nrows = min(RG_ROWS, H2 - h2_0);
+    const T *rows = x + ((size_t)n * H + (size_t)sf * h2_0) * W * c_mem;
+    const int row_elems = sf * W * c_mem;                // input elements behind one regrouped row
+    const int n_elems = nrows * row_elems;
     const size_t n_bytes = (size_t)n_elems * sizeof(T);
+    if (threadIdx.x < 16) {
+        const int ch = threadIdx.x, blk = ch / C, c = ch - blk * C;
+        const int dy = blk / sf, dx = blk - dy * sf;
+        src_off[ch] = blk < sf * sf ? (dy * W + dx) * c_mem + c : -1;
+    }
     if (((reinterpret_cast<uintptr_t>(rows) | n_bytes) & 15) == 0) {
         const uint4 *src = reinterpret_cast<const uint4 *>(rows);
         uint4 *dst = reinterpret_cast<uint4 *>(rg_smem);
@@ -778,23 +790,21 @@ __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, i
         for (int i = threadIdx.x; i < n_elems; i += blockDim.x) srow[i] = rows[i];
     }
     __syncthreads();
-    __nv_bfloat162 *orow = out + (size_t)blockIdx.x * WP * 8;
-    for (int e = threadIdx.x; e < WP * 8; e += blockDim.x) {
-        const int pair = e & 7, wp = e >> 3;
-        const int w2 = wp - pad_lo;
-        float v[2] = {0.f, 0.f};
-        if (w2 >= 0 && w2 < W2) {
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const int ch = 2 * pair + k;
-                const int blk = ch / C, c = ch - blk * C;
-                if (blk < sf * sf) {
-                    const int dy = blk / sf, dx = blk - dy * sf;
-                    v[k] = (float)srow[(dy * W + sf * w2 + dx) * c_mem + c];
-                }
+    __nv_bfloat162 *orow = out + ((size_t)n * H2 + h2_0) * WP * 8;
+    const int per_row = WP * 8;
+    const int step = sf * c_mem;                         // input elements between neighbouring regrouped pixels
+    for (int r = 0; r < nrows; ++r) {
+        const T *in = srow + (size_t)r * row_elems;
+        for (int e = threadIdx.x; e < per_row; e += blockDim.x) {
+            const int pair = e & 7, w2 = (e >> 3) - pad_lo;
+            float v0 = 0.f, v1 = 0.f;
+            if (w2 >= 0 && w2 < W2) {
+                const int o0 = src_off[2 * pair], o1 = src_off[2 * pair + 1];
+                if (o0 >= 0) v0 = (float)in[o0 + w2 * step];
+                if (o1 >= 0) v1 = (float)in[o1 + w2 * step];
             }
+            orow[(size_t)r * per_row + e] = __floats2bfloat162_rn(v0, v1);
         }
-        orow[e] = __floats2bfloat162_rn(v[0], v[1]);
     }
 }
 
@@ -844,8 +854,8 @@ cprune_status regroup_stem_input(const cprune_plan *plan, const void *x, int x_i
     const cprune_plan_info &i = plan->info;
     PatchGeometry g;
     if (!patch_geometry(i, &g) || !g.stem || !x || !scratch) return CPRUNE_ERR_INVALID_ARG;
-    const unsigned blocks = (unsigned)(i.N * g.He);
-    const size_t row_bytes = (size_t)g.sf * i.W * (x_is_f32 ? (size_t)i.C * 4 : (size_t)i.c_pad * 2);
+    const unsigned blocks = (unsigned)(i.N * ((g.He + RG_ROWS - 1) / RG_ROWS));
+    const size_t row_bytes = (size_t)RG_ROWS * g.sf * i.W * (x_is_f32 ? (size_t)i.C * 4 : (size_t)i.c_pad * 2);
     if (row_bytes > 48 * 1024) return CPRUNE_ERR_UNSUPPORTED;     // planning keeps such images off this path
     if (x_is_f32)
         CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3(blocks), dim3(256), row_bytes, st, (const float *)x, i.H, i.W, i.C, i.C, g.sf, g.pad_lo,
