@@ -112,20 +112,33 @@ __global__ void __launch_bounds__(256) fc_kernel(const bf16x8 *__restrict__ x, i
             }
         }
     }
+    // OB * NB = 32 partial sums per lane -> lane l ends up with the total of sum number l: at every halving step a lane
+    // keeps the half of the sums selected by one bit of its index and hands the other half to its partner (31 shuffles
+    // instead of 160)
+    static_assert(OB * NB == 32, "one total per lane");
+    float v[32];
 #pragma unroll
-    for (int q = 0; q < OB; ++q) {
-        const int o = o0 + q;
+    for (int q = 0; q < OB; ++q)
 #pragma unroll
-        for (int j = 0; j < NB; ++j) {
-            float v = acc[q][j];
-            for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-            if (lane == 0 && n0 + j < N) {
-                v = apply_act(v + b[o], act);
-                if (out_is_f32) {
-                    if (o < out) ((float *)y)[(size_t)(n0 + j) * out + o] = v;
-                } else {
-                    ((__nv_bfloat16 *)y)[(size_t)(n0 + j) * out_pad + o] = __float2bfloat16_rn(o < out ? v : 0.f);
-                }
+        for (int j = 0; j < NB; ++j) v[q * NB + j] = acc[q][j];
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool up = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            const float keep = up ? v[i + s] : v[i];
+            const float give = up ? v[i] : v[i + s];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, give, s);
+        }
+    }
+    {
+        const int o = o0 + lane / NB, n = n0 + lane % NB;
+        if (n < N) {
+            const float r = apply_act(v[0] + b[o], act);
+            if (out_is_f32) {
+                if (o < out) ((float *)y)[(size_t)n * out + o] = r;
+            } else {
+                ((__nv_bfloat16 *)y)[(size_t)n * out_pad + o] = __float2bfloat16_rn(o < out ? r : 0.f);
             }
         }
     }
