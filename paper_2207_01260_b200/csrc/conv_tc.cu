@@ -665,7 +665,7 @@ static cprune_status load_driver_entry_points() {
 }
 
 // Split-K finalize: y[m][k] = act(bias[k] + residual[m][k] + sum over slices of partial[s][m][k]),
-// slices added in index order (deterministic).  One thread per (output pixel, 8 filters).  With
+// slices added in a fixed order (deterministic).  Four threads per (conv pixel, 8 filters).  With
 // pool_q > 0 an output pixel is the maximum over its 2x2 window of conv pixels (image rows of pool_q
 // pixels; a pooled pixel j of an image covers conv pixels 2*(j / (pool_q/2))*pool_q + 2*(j % (pool_q/2)) + {0,1,pool_q,pool_q+1}).
 __global__ void __launch_bounds__(256) splitk_finalize_kernel(const float *__restrict__ partial, int splits, long long M,
@@ -674,38 +674,55 @@ __global__ void __launch_bounds__(256) splitk_finalize_kernel(const float *__res
                                                               bf16x8 *__restrict__ y) {
     pdl_trigger();
     pdl_wait();
-    const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long out_pixels = pool_q ? M / 4 : M;
-    if (e >= out_pixels * k8) return;
-    const long long mo = e / k8;
-    const int kg = (int)(e - mo * k8);
-    float bb[8], best[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) { bb[j] = __ldg(bias + kg * 8 + j); best[j] = -INFINITY; }
+    // Four lanes share one (conv pixel, 8 filters): lane L adds slices L, L + 4, ... in index order and the four sums are
+    // combined as (L0 + L1) + (L2 + L3): a fixed order, so the result does not depend on timing.  With a pool the four
+    // conv pixels of a window sit in four such lane groups (16 lanes per output).
     const int windows = pool_q ? 4 : 1;
+    const int lanes_per_out = 4 * windows;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long e = t / lanes_per_out;                      // output element group (pixel, 8 filters)
+    const int sub = (int)(t - e * lanes_per_out);
+    const int L = sub & 3, wdx = sub >> 2;
+    const long long out_pixels = pool_q ? M / 4 : M;
+    const bool valid = e < out_pixels * k8;                     // whole lane groups are valid or not (uniform shuffles below)
+    const long long ec = valid ? e : 0;
+    const long long mo = ec / k8;
+    const int kg = (int)(ec - mo * k8);
     const int hq = pool_q >> 1;
-    for (int wdx = 0; wdx < windows; ++wdx) {
-        long long m = mo;
-        if (pool_q) m = 2 * (mo / hq) * pool_q + 2 * (mo % hq) + (wdx & 1) + (wdx >> 1) * pool_q;
-        float f[8];
+    long long m = mo;
+    if (pool_q) m = 2 * (mo / hq) * pool_q + 2 * (mo % hq) + (wdx & 1) + (wdx >> 1) * pool_q;
+    float f[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) f[j] = bb[j];
-        for (int sidx = 0; sidx < splits; ++sidx) {
-            const float4 *src = (const float4 *)(partial + ((size_t)sidx * M + m) * k_alloc + kg * 8);
-            const float4 a = __ldg(src), b = __ldg(src + 1);
-            f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
-            f[4] += b.x; f[5] += b.y; f[6] += b.z; f[7] += b.w;
-        }
-        if (res) {
-            float rf[8];
-            unpack8(ldg8(res + m * k8 + kg), rf);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) f[j] += rf[j];
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) best[j] = fmaxf(best[j], apply_act(f[j], act));
+    for (int j = 0; j < 8; ++j) f[j] = 0.f;
+    for (int sidx = L; sidx < splits; sidx += 4) {
+        const float4 *src = (const float4 *)(partial + ((size_t)sidx * M + m) * k_alloc + kg * 8);
+        const float4 a = __ldg(src), b = __ldg(src + 1);
+        f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+        f[4] += b.x; f[5] += b.y; f[6] += b.z; f[7] += b.w;
     }
-    y[e] = pack8(best);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        f[j] += __shfl_xor_sync(0xffffffffu, f[j], 1);
+        f[j] += __shfl_xor_sync(0xffffffffu, f[j], 2);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] += __ldg(bias + kg * 8 + j);
+    if (res) {
+        float rf[8];
+        unpack8(ldg8(res + m * k8 + kg), rf);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] += rf[j];
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) f[j] = apply_act(f[j], act);
+    if (pool_q) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            f[j] = fmaxf(f[j], __shfl_xor_sync(0xffffffffu, f[j], 4));
+            f[j] = fmaxf(f[j], __shfl_xor_sync(0xffffffffu, f[j], 8));
+        }
+    }
+    if (valid && sub == 0) y[e] = pack8(f);
 }
 
 // 128 x 128 identity in bf16: the filter-side operand of the residual blocks (see the producer).
@@ -1046,7 +1063,7 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     }
     CPRUNE_LAUNCH_CHECK("conv_tc_kernel");
     if (split) {
-        const long long elems = (plan->fused_pool ? p.M / 4 : p.M) * (i.k_pad / 8);
+        const long long elems = (plan->fused_pool ? p.M / 4 : p.M) * (i.k_pad / 8) * (plan->fused_pool ? 16 : 4);   // threads
         CPRUNE_CUDA_CHECK(launch_chained(splitk_finalize_kernel, dim3((unsigned)ceil_div(elems, 256)), dim3(256), 0, st, (const float *)partial,
                                          plan->splits, p.M, i.k_alloc, i.k_pad / 8, b, (const bf16x8 *)res, plan->opts.activation,
                                          plan->fused_pool ? i.Q : 0, (bf16x8 *)y));
