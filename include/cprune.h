@@ -148,7 +148,9 @@ typedef struct {
 /* Host only; launches nothing.  opts == NULL means bias + ReLU, no residual, no pool, AUTO.
  * Plans are cached: an identical (shape, opts) key returns the same handle with its reference
  * count raised.  groups must be 1 or C (depthwise; then K == C and R == S == 3).
- * Errors: INVALID_ARG (non-positive extents, output extent < 1, pool on odd P/Q), UNSUPPORTED. */
+ * The pool option (paper Sec. 3.4: a task is the fused subgraph) is applied to the activated result:
+ * CPRUNE_POOL_MAX2X2 needs even P and Q; CPRUNE_POOL_MAX3X3S2 (3x3, stride 2, pad 1) takes any extent.
+ * Errors: INVALID_ARG (non-positive extents, output extent < 1, 2x2 pool on odd P/Q), UNSUPPORTED. */
 cprune_status cprune_task_plan(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int groups,
                                const cprune_task_opts *opts, cprune_plan **out);
 cprune_status cprune_plan_query(const cprune_plan *plan, cprune_plan_info *out /* host */);
@@ -161,7 +163,9 @@ cprune_status cprune_cache_stats(int *n_plans, long long *n_hits);
 
 /* One-time layout change of a (pruned) layer's parameters for its plan:
  * w float32 [K][C/groups][R][S] -> bfloat16 (round to nearest even) [k_alloc][R][S][c_pad] with zero
- * padding (depthwise: [R][S][c_pad]); b float32 [K] (NULL = zeros) -> float32 [k_alloc] zero padded.
+ * padding (depthwise: [R][S][c_pad]; stems that the plan runs on a regrouped input: the plan's own
+ * order of taps and channels); b float32 [K] (NULL = zeros) -> float32 [k_alloc] zero padded.
+ * The packed layout belongs to the plan: pack with the plan the task will run with.
  * All pointers device; w_packed needs packed_weight_bytes, b_packed packed_bias_bytes. */
 cprune_status cprune_pack_weights(const cprune_plan *plan, const float *w, const float *b, void *w_packed,
                                   float *b_packed, void *stream);
@@ -169,8 +173,10 @@ cprune_status cprune_pack_weights(const cprune_plan *plan, const float *w, const
 /* Runs one task: y = pool(act(conv(x, w) + b + residual)).
  *   x         device, bf16 [N][H][W][c_pad]          residual  device, bf16 [N][P][Q][k_pad] or NULL
  *   y         device, bf16 [N][out_h][out_w][k_pad]  workspace device, workspace_bytes (may be NULL if 0)
- * Enqueue only (at most two launches), no allocation, no synchronisation.  Pointers must be 16-byte
- * aligned.  Errors: INVALID_ARG (null pointer, residual mismatch with the plan), CUDA. */
+ * The workspace holds what the plan needs besides x and y: float32 partial sums of a split reduction,
+ * the unpooled result when the pool runs as a separate pass, the regrouped input of a stem.
+ * Enqueue only (at most three launches), no allocation, no synchronisation.  Pointers must be 16-byte
+ * aligned.  Errors: INVALID_ARG (null pointer, missing workspace, residual mismatch with the plan), CUDA. */
 cprune_status cprune_task_run(cprune_plan *plan, const void *x, const void *w_packed, const float *b_packed,
                               const void *residual, void *y, void *workspace, void *stream);
 
