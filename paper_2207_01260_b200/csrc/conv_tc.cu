@@ -835,6 +835,10 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
             if ((long long)tiles_m * tiles_n >= 148) break;
             tiles_n = next;
         }
+        if (const char *e = getenv("CPRUNE_TC_TILES_N")) {     // measurement override
+            const int v = atoi(e);
+            if (v >= (k16 + 255) / 256 && v <= 16) tiles_n = v;
+        }
         // with several filter tiles every tile must end on a 64-filter boundary: the staged stores
         // are 64 filters wide and only the tensor's own edge clips them
         FT = round_up((k16 + tiles_n - 1) / tiles_n, tiles_n > 1 ? 64 : 16);
