@@ -66,6 +66,17 @@ def test_plan_shapes_and_families(cp):
     # the CUDA-core family does not fuse it: the unpooled output goes to the workspace
     p = cp.cprune_task_plan(128, 45, 32, 32, 58, 3, 3, 1, 1, pool="max2x2", kernel="direct")
     assert (p.out_h, p.out_w) == (16, 16) and p.workspace_bytes == 128 * 32 * 32 * 64 * 2
+    # a pointwise stride-1 task with many pixels is planned as a flat matrix product: tiles of 128 or 256 pixels
+    f = cp.cprune_task_plan(64, 24, 56, 56, 108, 1, 1, 1, 0, activation="relu6")
+    assert f.variant == 1 and f.tile_m in (128, 256) and f.tiles_m == -(-64 * 56 * 56 // f.tile_m) and f.workspace_bytes == 0
+    # the ResNet stem with its 3x3 stride-2 pool: pooled output extent, pool fused (no unpooled copy in the workspace,
+    # only the regrouped input), tiles around whole pooling windows
+    sp = cp.cprune_task_plan(64, 3, 224, 224, 64, 7, 7, 2, 3, pool="max3x3s2")
+    assert (sp.P, sp.Q, sp.out_h, sp.out_w) == (112, 112, 56, 56) and sp.variant == 1
+    assert sp.workspace_bytes == s.workspace_bytes
+    # the same pool on a task the patch kernel cannot fuse it into runs as a separate pass over an unpooled copy
+    sq = cp.cprune_task_plan(2, 16, 30, 30, 24, 3, 3, 1, 1, pool="max3x3s2")
+    assert (sq.out_h, sq.out_w) == (15, 15) and sq.workspace_bytes >= 2 * 30 * 30 * 24 * 2
     # every pruned filter count gets a legal tile: N tile a multiple of 16 within the accumulator
     for K in range(64, 513, 7):
         p = cp.cprune_task_plan(64, 256, 14, 14, K, 3, 3, 1, 1)
