@@ -58,6 +58,8 @@ struct PatchParams {
     int patch_box_bytes;   // bytes one patch load delivers
     int w_stage_bytes;     // shared memory of one filter stage (FT rows, rounded up to 1024 bytes)
     int rb16;              // bytes per pixel row in shared memory / 16: 8 (64 channels) or 2 (16 channels, regrouped stems)
+    int dense;             // the staged tile is [slot][k_pad] as in memory and leaves by one bulk copy (flat tasks, one filter tile)
+    int stage_bytes;       // shared memory of one staging buffer
     const float *bias;
     const __nv_bfloat16 *res;
     __nv_bfloat16 *y;
@@ -138,6 +140,7 @@ __device__ __forceinline__ void tile_origin(const PatchParams &p, int tm, int &n
     q0 = tx * p.step_w + p.org;
 }
 
+template <bool DENSE>
 __global__ void __launch_bounds__(PK_THREADS, 1)
 conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res, const PatchParams p) {
@@ -151,7 +154,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const uint32_t patch0 = base;
     const uint32_t w0 = patch0 + (uint32_t)p.pstages * (uint32_t)p.patch_bytes;
     const uint32_t staging0 = w0 + (uint32_t)p.wstages * w_bytes;
-    const uint32_t stage_buf_bytes = (uint32_t)p.MT * PK_BLOCK_BYTES;
+    const uint32_t stage_buf_bytes = (uint32_t)p.stage_bytes;
     const uint32_t ctrl0 = staging0 + (uint32_t)p.staging_bufs * stage_buf_bytes;
     uint8_t *ctrl = smem + (ctrl0 - base);
     auto pfull = [&](int s) { return ctrl0 + 8u * s; };
@@ -343,7 +346,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // the shared-memory offsets of their nine window slots are worked out once
         uint32_t win_off[2][9];
         int win_pi[2] = {0, 0}, win_pj[2] = {0, 0};
-        if (p.pool == 2) {
+        if (!DENSE && p.pool == 2) {
             const int tpc = (p.TW - 1) >> 1;
 #pragma unroll
             for (int it = 0; it < 2; ++it) {
@@ -370,7 +373,18 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             mbar_expect_tx(res_full(b), (uint32_t)(p.TH * p.Wp * 128));
             tma_load_4d(staging0 + b * stage_buf_bytes, &tm_res, res_full(b), nt_ * p.FT + g_ * 64, q0_, p0_, n_);
         };
-        if (with_res && store_thread && (int)blockIdx.x < total_items) load_residual(blockIdx.x, 0, 0);
+        // dense staging: the residual of tile item_ (tiles_n == 1, one row of tiles) is one contiguous range as well
+        auto load_residual_dense = [&](int item_, uint32_t counter) {
+            const int q0_ = item_ * p.step_w;
+            const uint32_t bytes = (uint32_t)min(p.TW, p.Q - q0_) * (uint32_t)p.k_pad * 2u;
+            const uint32_t b = counter & 1u;
+            mbar_expect_tx(res_full(b), bytes);
+            bulk_load(staging0 + b * stage_buf_bytes, p.res + (size_t)q0_ * p.k_pad, bytes, res_full(b));
+        };
+        if (with_res && store_thread && (int)blockIdx.x < total_items) {
+            if constexpr (DENSE) load_residual_dense(blockIdx.x, 0);
+            else load_residual(blockIdx.x, 0, 0);
+        }
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
             int tm = item, nt = 0;
             if (p.tiles_n > 1) { tm = item / p.tiles_n; nt = item - tm * p.tiles_n; }
@@ -384,6 +398,73 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.MT * p.FT);
+            if constexpr (DENSE) {
+                // Flat task with one filter tile: the tile's output is ONE contiguous range of y (slot-major, k_pad filters
+                // per slot).  It is staged in exactly that layout and leaves by a single bulk copy; a residual arrives the
+                // same way.  (Rows of k_pad * 2 bytes: the 16-byte pieces of eight neighbouring slots fall in distinct banks.)
+                const uint32_t b = group_counter & 1u;
+                uint8_t *buf = smem + (staging0 - base) + b * stage_buf_bytes;
+                const uint32_t pitch = (uint32_t)p.k_pad * 2u;
+                if (with_res) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), (group_counter >> 1) & 1u, abort_flag, p.status, false));
+                    if (!ok) break;
+                }
+                for (int g = 0; g < groups; ++g) {
+                    const int ch = g * 64 + half * 32;
+                    for (int mb = 0; mb < p.MT; ++mb) {
+                        uint8_t *row = buf + (uint32_t)(mb * 128 + trow) * pitch;
+                        uint32_t v[32];
+#pragma unroll
+                        for (int sb = 0; sb < 2; ++sb)
+                            if (ch + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(mb * p.FT + ch + sb * 16), v + sb * 16);
+                        bf16x8 rv[4];
+                        if (with_res) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (ch + j * 8 < p.k_pad) rv[j] = *(const bf16x8 *)(row + (ch + j * 8) * 2);
+                        }
+                        tmem_ld_wait();
+                        if (g == groups - 1 && mb == p.MT - 1) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(tempty(acc));
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int c = ch + q * 8;
+                            if (c < p.k_pad) {
+                                float f[8];
+                                const float4 b0 = __ldg((const float4 *)(p.bias + c));
+                                const float4 b1 = __ldg((const float4 *)(p.bias + c + 4));
+                                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[q * 8 + j]) + bb[j];
+                                if (with_res) {
+                                    float rf[8];
+                                    unpack8(rv[q], rf);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) f[j] += rf[j];
+                                }
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) f[j] = fminf(fmaxf(f[j], act_lo), act_hi);
+                                *(bf16x8 *)(row + c * 2) = pack8(f);
+                            }
+                        }
+                    }
+                }
+                fence_async_smem();
+                // the other buffer, written next, was last read by the previous tile's store
+                if (store_thread) tma_store_wait_read<0>();
+                ok = epi_sync();
+                if (!ok) break;
+                if (store_thread) {
+                    const int rows = min(p.TW, p.Q - q0);
+                    bulk_store(p.y + (size_t)q0 * p.k_pad, staging0 + b * stage_buf_bytes, (uint32_t)rows * pitch);
+                    tma_store_commit();
+                    if (with_res && item + (int)gridDim.x < total_items) load_residual_dense(item + gridDim.x, group_counter + 1);
+                }
+                ++group_counter;
+            } else {
             for (int g = 0; g < groups && ok; ++g) {
                 const uint32_t boff = (p.staging_bufs == 2 ? (group_counter & 1u) : 0u) * stage_buf_bytes;
                 uint8_t *buf = smem + (staging0 - base) + boff;
@@ -526,6 +607,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     if (!ok) break;
                 }
                 ++group_counter;
+            }
             }
             if (p.acc_bufs == 2) { if (++acc == 2) { acc = 0; acc_phase ^= 1u; } }
             else acc_phase ^= 1u;
@@ -683,12 +765,26 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             if (patch_bytes < Wp * (TH + g.kR - 1) * RB) continue;
             // patch ring depth: two stages; up to four when the task has that many channel blocks and the patches are
             // small (1x1 tasks), because each load's latency is otherwise exposed
-            int pstages = 2;
-            if (cblks > 2 && patch_bytes <= 32 * 1024) pstages = cblks < PK_MAX_PATCH_STAGES ? cblks : PK_MAX_PATCH_STAGES;
+            // (flat tasks: a tile is little work, and a patch load's latency under a stream of output writes is several
+            // tiles long, so the ring is as deep as fits)
+            int ps_max = 2;
+            if (cblks > 2 && patch_bytes <= 32 * 1024) ps_max = cblks < PK_MAX_PATCH_STAGES ? cblks : PK_MAX_PATCH_STAGES;
+            const char *force_ps = getenv("CPRUNE_PATCH_PSTAGES");      // measurement override
+            if (g.flat) ps_max = force_ps ? atoi(force_ps) : PK_MAX_PATCH_STAGES;
+            if (ps_max < 2) ps_max = 2;
+            if (ps_max > PK_MAX_PATCH_STAGES) ps_max = PK_MAX_PATCH_STAGES;
+          for (int pstages = ps_max; pstages >= 2; --pstages) {
             const int fixed = 1024 + pstages * patch_bytes + PK_CTRL_BYTES;
             const int budget = 227 * 1024 - fixed;
             const int sb_max = 2, sb_min = 1;
             const int w_stage = round_up(FT * RB, 1024);
+            // flat tasks with one filter tile stage the tile as it lies in memory (k_pad filters per pixel) when that fits
+            // and the pixel pitch is an odd number of 16-byte pieces (no bank conflicts between neighbouring pixels;
+            // 32-byte pixels conflict two-way and still gain, measured)
+            const char *force_dense = getenv("CPRUNE_PATCH_DENSE");     // measurement override: 0 = never
+            const int dense_bytes = round_up(128 * MT * i.k_pad * 2, 1024);
+            const int dense = g.flat && tiles_n == 1 && (((i.k_pad >> 3) & 1) || i.k_pad == 16) && dense_bytes <= 40 * 1024 && !(force_dense && force_dense[0] == '0');
+            const int stage_bytes = dense ? dense_bytes : MT * PK_BLOCK_BYTES;
             int staging_bufs = sb_max, wstages = 0, resident = 0;
             // resident filters when the whole set of this filter tile fits
             // (with a residual, only beside two staging buffers: with one buffer the residual of a group can only be
@@ -697,26 +793,29 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             const int sb_res_min = (plan->opts.residual && !(force_res && force_res[0] == '1')) ? 2 : sb_min;
             if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES && !(force_res && force_res[0] == '0')) {
                 for (int sb = sb_max; sb >= sb_res_min && !resident; --sb)
-                    if (RS * cblks * w_stage + sb * MT * PK_BLOCK_BYTES <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
+                    if (RS * cblks * w_stage + sb * stage_bytes <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
             }
             if (!resident) {
                 staging_bufs = sb_max;
-                wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / w_stage;
+                wstages = (budget - staging_bufs * stage_bytes) / w_stage;
                 if (wstages < 3 && sb_min < sb_max) {
                     staging_bufs = sb_min;
-                    wstages = (budget - staging_bufs * MT * PK_BLOCK_BYTES) / w_stage;
+                    wstages = (budget - staging_bufs * stage_bytes) / w_stage;
                 }
                 if (wstages < 3) continue;
                 if (wstages > 8) wstages = 8;
             }
+            if (dense && staging_bufs != 2) continue;
             const long long tiles = (long long)g.vN * tiles_per_img * tiles_n;
             const double waves = (double)((tiles + 147) / 148);
             double t = waves * tile_cycles(MT, FT, RS, cblks, ksteps_last, RB, Wp, TH, g.kR, resident != 0, acc_bufs);
             if (resident) t += RS * cblks * FT;    // one-time filter load
             if (t < best) {
                 best = t;
-                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org, pstages};
+                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org, pstages, dense, stage_bytes};
             }
+            break;      // the deepest ring that fits
+          }
         }
       }
     }
@@ -747,7 +846,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     const int ksteps = (cblks - 1) * 4 + ksteps_last;
     i.padded_flops = 2.0 * (double)i.tiles_m * i.tile_m * (double)i.k_alloc * RS * ksteps * 16.0;
     plan->smem_bytes = 1024 + bt.pstages * bt.patch_bytes + bt.wstages * round_up(bt.FT * RB, 1024) +
-                       bt.staging_bufs * bt.MT * PK_BLOCK_BYTES + PK_CTRL_BYTES;
+                       bt.staging_bufs * bt.stage_bytes + PK_CTRL_BYTES;
     return CPRUNE_OK;
 }
 
@@ -947,7 +1046,8 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     {
         std::lock_guard<std::mutex> lock(attr_mu);
         if (!attr_set) {
-            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             attr_set = true;
         }
     }
@@ -965,6 +1065,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     p.patch_bytes = t.patch_bytes;
     p.patch_box_bytes = Wp * (t.TH + g.kR - 1) * 128;
     p.rb16 = 8;
+    p.dense = t.dense; p.stage_bytes = t.stage_bytes;
     p.w_stage_bytes = t.FT * 128;
     p.bias = b;
     p.res = (const __nv_bfloat16 *)res;
@@ -977,7 +1078,10 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
     const int grid = total < sms ? total : sms;
-    CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
+    if (t.dense)
+        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<true>, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
+    else
+        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<false>, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     return CPRUNE_OK;
 }
 

@@ -15,6 +15,8 @@ struct PatchTiling {
     int MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes;
     int TW, tiles_w, step_h, step_w, org;   // tile width, tiles per image row, distance between tiles, origin offset
     int pstages;                            // depth of the patch ring
+    int dense;                              // flat tasks: a tile's output is staged as it lies in memory and stored by one bulk copy
+    int stage_bytes;                        // shared memory of one staging buffer
 };
 
 struct cprune_plan {
