@@ -178,6 +178,12 @@ def test_pointwise_tasks_as_flat_matrix_products(cp):
     check_task(cp, 3, 108, 57, 59, 24, 1, 1, 0, act="none", with_res=True, kernel="tensor")
     check_task(cp, 5, 72, 40, 41, 300, 1, 1, 0, act="relu", kernel="tensor")
     check_task(cp, 64, 320, 7, 7, 1280, 1, 1, 0, act="relu6", kernel="tensor")
+    # one filter tile and a pixel pitch of an odd number of 16-byte pieces (or 32 bytes): the tile is staged as it lies
+    # in memory and leaves by one bulk copy (one and two 64-filter groups, with and without residual, ragged last tile)
+    check_task(cp, 6, 16, 50, 53, 72, 1, 1, 0, act="relu6", kernel="tensor")
+    check_task(cp, 6, 32, 47, 50, 16, 1, 1, 0, act="none", kernel="tensor")
+    check_task(cp, 4, 150, 45, 46, 40, 1, 1, 0, act="relu6", with_res=True, kernel="tensor")
+    check_task(cp, 4, 48, 45, 46, 133, 1, 1, 0, act="relu", with_res=True, kernel="tensor")
 
 
 def test_stems_on_the_patch_kernel(cp):
