@@ -45,7 +45,8 @@ constexpr int PK_FIRST_EPI = 4;
 constexpr int PK_MMA_WARP2 = 12;         // issues for the second accumulator block when MT = 2
 constexpr int PK_MAX_WSTAGES = 32;
 constexpr int PK_MAX_PATCH_STAGES = 4;   // patch ring: 2 stages, more for tasks with small patches and several channel blocks
-constexpr int PK_CTRL_BYTES = 3072;      // barriers (1 KB) + slot table (2 KB)
+constexpr int PK_CTRL_BYTES = 5120;      // barriers (1 KB) + slot table (2 KB) + bias (2 KB)
+constexpr int PK_BIAS_FLOATS = 512;      // the task's bias is kept in shared memory when it has at most this many filters
 constexpr int PK_BLOCK_BYTES = 16384;    // staged block: 128 slots x 64 filters bf16
 
 struct PatchParams {
@@ -184,6 +185,13 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         if (l < p.wstages) { mbar_init(wfull(l), 1); mbar_init(wempty(l), p.MT); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // the bias (written when the task was packed, not by the preceding kernel) in shared memory: a read costs the
+    // epilogue a fraction of what the same read through L1 does
+    float *bias_s = (float *)(ctrl + 3072);
+    const int k_all = p.tiles_n * p.FT;
+    const bool bias_staged = k_all <= PK_BIAS_FLOATS;
+    for (int e = threadIdx.x; e < k_all && bias_staged; e += PK_THREADS) bias_s[e] = __ldg(p.bias + e);
+    const float *bias_src = bias_staged ? bias_s : p.bias;
     // slot table: which accumulator rows hold real output pixels and where they go
     for (int e = threadIdx.x; e < 256 && p.pool == 1; e += PK_THREADS) {
         int2 v = make_int2(-1, 0);
@@ -434,8 +442,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                             const int c = ch + q * 8;
                             if (c < p.k_pad) {
                                 float f[8];
-                                const float4 b0 = __ldg((const float4 *)(p.bias + c));
-                                const float4 b1 = __ldg((const float4 *)(p.bias + c + 4));
+                                const float4 b0 = *(const float4 *)(bias_src + c);
+                                const float4 b1 = *(const float4 *)(bias_src + c + 4);
                                 const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[q * 8 + j]) + bb[j];
@@ -500,8 +508,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
                                 float f[8];
-                                const float4 b0 = __ldg((const float4 *)(p.bias + k0 + c0 + h * 8));
-                                const float4 b1 = __ldg((const float4 *)(p.bias + k0 + c0 + h * 8 + 4));
+                                const float4 b0 = *(const float4 *)(bias_src + k0 + c0 + h * 8);
+                                const float4 b1 = *(const float4 *)(bias_src + k0 + c0 + h * 8 + 4);
                                 const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[sb * 16 + h * 8 + j]) + bb[j];
