@@ -39,10 +39,12 @@
 
 namespace cprune {
 
-constexpr int PK_THREADS = 13 * 32;
+constexpr int PK_THREADS = 13 * 32;       // general kernel: 5 role warps + 8 epilogue warps
+constexpr int PK_THREADS_DENSE = 21 * 32; // dense-staging kernel: 16 epilogue warps (its epilogue bounds the tile; it needs few registers)
+__host__ __device__ constexpr int pk_epi_warps(bool dense) { return dense ? 16 : 8; }
 constexpr int PK_MMA_WARP = 3;
 constexpr int PK_FIRST_EPI = 4;
-constexpr int PK_MMA_WARP2 = 12;         // issues for the second accumulator block when MT = 2
+// (the warp after the epilogue warps issues for the second accumulator block when MT = 2)
 constexpr int PK_MAX_WSTAGES = 32;
 constexpr int PK_MAX_PATCH_STAGES = 4;   // patch ring: 2 stages, more for tasks with small patches and several channel blocks
 constexpr int PK_CTRL_BYTES = 5120;      // barriers (1 KB) + slot table (2 KB) + bias (2 KB)
@@ -142,10 +144,12 @@ __device__ __forceinline__ void tile_origin(const PatchParams &p, int tm, int &n
 }
 
 template <bool DENSE>
-__global__ void __launch_bounds__(PK_THREADS, 1)
+__global__ void __launch_bounds__(DENSE ? PK_THREADS_DENSE : PK_THREADS, 1)
 conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res, const PatchParams p) {
     extern __shared__ uint8_t smem_raw[];
+    constexpr int EPI_WARPS = pk_epi_warps(DENSE);
+    constexpr int MMA_WARP2 = PK_FIRST_EPI + EPI_WARPS;
     pdl_trigger();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -180,8 +184,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     if (threadIdx.x < 32) {
         const int l = threadIdx.x;
         if (l < p.pstages) { mbar_init(pfull(l), 1); mbar_init(pempty(l), p.MT); }
-        if (l < 2) { mbar_init(tfull(l), p.MT); mbar_init(tempty(l), 8); mbar_init(res_full(l), 1); }
-        if (l == 2) { mbar_init(epi_bar, 8); *abort_flag = 0; }
+        if (l < 2) { mbar_init(tfull(l), p.MT); mbar_init(tempty(l), EPI_WARPS); mbar_init(res_full(l), 1); }
+        if (l == 2) { mbar_init(epi_bar, EPI_WARPS); *abort_flag = 0; }
         if (l < p.wstages) { mbar_init(wfull(l), 1); mbar_init(wempty(l), p.MT); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -190,10 +194,10 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     float *bias_s = (float *)(ctrl + 3072);
     const int k_all = p.tiles_n * p.FT;
     const bool bias_staged = k_all <= PK_BIAS_FLOATS;
-    for (int e = threadIdx.x; e < k_all && bias_staged; e += PK_THREADS) bias_s[e] = __ldg(p.bias + e);
+    for (int e = threadIdx.x; e < k_all && bias_staged; e += blockDim.x) bias_s[e] = __ldg(p.bias + e);
     const float *bias_src = bias_staged ? bias_s : p.bias;
     // slot table: which accumulator rows hold real output pixels and where they go
-    for (int e = threadIdx.x; e < 256 && p.pool == 1; e += PK_THREADS) {
+    for (int e = threadIdx.x; e < 256 && p.pool == 1; e += blockDim.x) {
         int2 v = make_int2(-1, 0);
         {
             const int hq = p.Q >> 1;
@@ -263,7 +267,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 }
             }
         }
-    } else if (warp == PK_MMA_WARP || warp == PK_MMA_WARP2) {
+    } else if (warp == PK_MMA_WARP || warp == MMA_WARP2) {
         // ------------------------------------------------------------------ MMA issue
         // tcgen05.mma issue is close to synchronous (about two instructions may be pending, measured), so the
         // bookkeeping between taps would leave the tensor pipe idle if one warp issued everything: with MT = 2
@@ -418,27 +422,21 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     if (!ok) break;
                 }
                 for (int g = 0; g < groups; ++g) {
-                    const int ch = g * 64 + half * 32;
+                    const int ch = g * 64 + half * 16;           // this warp's 16 filters of the group (16 epilogue warps)
+                    if (ch >= p.k_pad) continue;
                     for (int mb = 0; mb < p.MT; ++mb) {
                         uint8_t *row = buf + (uint32_t)(mb * 128 + trow) * pitch;
-                        uint32_t v[32];
-#pragma unroll
-                        for (int sb = 0; sb < 2; ++sb)
-                            if (ch + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(mb * p.FT + ch + sb * 16), v + sb * 16);
-                        bf16x8 rv[4];
+                        uint32_t v[16];
+                        tmem_ld16(t_row + (uint32_t)(mb * p.FT + ch), v);
+                        bf16x8 rv[2];
                         if (with_res) {
 #pragma unroll
-                            for (int j = 0; j < 4; ++j)
+                            for (int j = 0; j < 2; ++j)
                                 if (ch + j * 8 < p.k_pad) rv[j] = *(const bf16x8 *)(row + (ch + j * 8) * 2);
                         }
                         tmem_ld_wait();
-                        if (g == groups - 1 && mb == p.MT - 1) {
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(tempty(acc));
-                        }
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
+                        for (int q = 0; q < 2; ++q) {
                             const int c = ch + q * 8;
                             if (c < p.k_pad) {
                                 float f[8];
@@ -460,6 +458,10 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                         }
                     }
                 }
+                // every warp has read what it needs of the accumulator (a warp without filters in the last group too)
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty(acc));
                 fence_async_smem();
                 // the other buffer, written next, was last read by the previous tile's store
                 if (store_thread) tma_store_wait_read<0>();
@@ -1087,7 +1089,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
     const int grid = total < sms ? total : sms;
     if (t.dense)
-        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<true>, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
+        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<true>, dim3(grid), dim3(PK_THREADS_DENSE), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     else
         CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<false>, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     return CPRUNE_OK;
