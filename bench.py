@@ -257,7 +257,7 @@ def main():
         per_task = net_task_times(cp, net, table, x, reps=5)
         # the tensor family has two kernels; the roofline object describes the one that takes more of the step
         tens_all = [t for t in per_task if t["kernel"] == "tensor"]
-        by_variant = {v: [t for t in tens_all if t["variant"] == v] for v in (0, 1)}
+        by_variant = {v: [t for t in tens_all if min(t["variant"], 1) == v] for v in (0, 1)}   # variants 1 and 2: the patch kernel
         top = max((0, 1), key=lambda v: sum(t["ms"] for t in by_variant[v]))
         tens = by_variant[top]
         tens_name = "conv_patch_kernel" if top == 1 else "conv_tc_kernel"

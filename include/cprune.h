@@ -142,7 +142,9 @@ typedef struct {
     double algorithmic_bytes; /* bf16 x + bf16 y (+ bf16 residual) + bf16 w + fp32 b, each once */
     double padded_flops;      /* flops the chosen kernel issues, including channel and tile padding */
     int variant;              /* tensor family: 0 = operands gathered per filter tap (im2col loads), 1 = the input patch
-                                 of a tile stays in shared memory and every tap reads it (stride-1 tasks, stems) */
+                                 of a tile stays in shared memory and every tap reads it (stride-1 tasks, stems),
+                                 2 = as 1, for 1x1 tasks whose output tile is one contiguous range of y: staged as it
+                                 lies in memory and stored by a single bulk copy */
 } cprune_plan_info;
 
 /* Host only; launches nothing.  opts == NULL means bias + ReLU, no residual, no pool, AUTO.

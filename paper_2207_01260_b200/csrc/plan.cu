@@ -77,7 +77,7 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     }
     if (st != CPRUNE_OK) { delete pl; return st; }
     i.kernel = family;
-    i.variant = (family == CPRUNE_KERNEL_TENSOR && pl->patch) ? 1 : 0;
+    i.variant = (family == CPRUNE_KERNEL_TENSOR && pl->patch) ? (pl->pt.dense ? 2 : 1) : 0;
     const double rs = (double)i.R * i.S;
     const int s_packed = (family == CPRUNE_KERNEL_TENSOR && pl->s_packed > 0) ? pl->s_packed : i.S;
     i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * s_packed * i.c_pad * 2;

@@ -180,10 +180,11 @@ def test_pointwise_tasks_as_flat_matrix_products(cp):
     check_task(cp, 64, 320, 7, 7, 1280, 1, 1, 0, act="relu6", kernel="tensor")
     # one filter tile and a pixel pitch of an odd number of 16-byte pieces (or 32 bytes): the tile is staged as it lies
     # in memory and leaves by one bulk copy (one and two 64-filter groups, with and without residual, ragged last tile)
-    check_task(cp, 6, 16, 50, 53, 72, 1, 1, 0, act="relu6", kernel="tensor")
-    check_task(cp, 6, 32, 47, 50, 16, 1, 1, 0, act="none", kernel="tensor")
-    check_task(cp, 4, 150, 45, 46, 40, 1, 1, 0, act="relu6", with_res=True, kernel="tensor")
-    check_task(cp, 4, 48, 45, 46, 133, 1, 1, 0, act="relu", with_res=True, kernel="tensor")
+    for case in ((12, 16, 50, 53, 72, "relu6", False), (6, 32, 47, 50, 16, "none", False), (4, 150, 45, 46, 40, "relu6", True),
+                 (8, 48, 45, 46, 133, "relu", True)):
+        N, C, H, W, K, act, res = case
+        plan = check_task(cp, N, C, H, W, K, 1, 1, 0, act=act, with_res=res, kernel="tensor")
+        assert plan.variant == 2, case
 
 
 def test_stems_on_the_patch_kernel(cp):
