@@ -217,6 +217,7 @@ def test_maxpool_3x3_stride_2(cp, case):
     (64, 512, 7, 7, 358, 3, 1, 1, 1, "relu", False, None),             # stage 4 (im2col kernel)
     (64, 64, 56, 56, 89, 3, 2, 1, 1, "relu", False, None),             # stride-2 3x3 (im2col kernel)
     (64, 16, 112, 112, 72, 1, 1, 0, 1, "relu6", False, None),          # MobileNetV2 expand (flat matrix product)
+    (64, 108, 56, 56, 24, 1, 1, 0, 1, "none", True, None),             # MobileNetV2 project + residual (flat, one bulk store per tile)
     (64, 72, 112, 112, 72, 3, 2, 1, 72, "relu6", False, None)])        # depthwise, stride 2
 def test_full_size_tasks_on_sampled_outputs(cp, case):
     N, C, H, W, K, R, stride, pad, groups, act, with_res, pool = case
