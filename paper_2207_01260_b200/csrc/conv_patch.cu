@@ -41,6 +41,11 @@ namespace cprune {
 
 constexpr int PK_THREADS = 13 * 32;       // general kernel: 5 role warps + 8 epilogue warps
 constexpr int PK_THREADS_DENSE = 21 * 32; // dense-staging kernel: 16 epilogue warps (its epilogue bounds the tile; it needs few registers)
+constexpr int PK_POOL_WARPS = 4;          // 3x3-pool kernel: these warps pool the staged tile while the epilogue warps stage the next one
+constexpr int PK_THREADS_POOL3 = (13 + PK_POOL_WARPS) * 32;
+// kernel instantiations
+constexpr int PK_GENERAL = 0, PK_DENSE = 1, PK_POOL3 = 2;
+__host__ __device__ constexpr int pk_threads(int mode) { return mode == PK_DENSE ? PK_THREADS_DENSE : (mode == PK_POOL3 ? PK_THREADS_POOL3 : PK_THREADS); }
 __host__ __device__ constexpr int pk_epi_warps(bool dense) { return dense ? 16 : 8; }
 constexpr int PK_MMA_WARP = 3;
 constexpr int PK_FIRST_EPI = 4;
@@ -143,11 +148,13 @@ __device__ __forceinline__ void tile_origin(const PatchParams &p, int tm, int &n
     q0 = tx * p.step_w + p.org;
 }
 
-template <bool DENSE>
-__global__ void __launch_bounds__(DENSE ? PK_THREADS_DENSE : PK_THREADS, 1)
+template <int MODE>
+__global__ void __launch_bounds__(pk_threads(MODE), 1)
 conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_res, const PatchParams p) {
     extern __shared__ uint8_t smem_raw[];
+    constexpr bool DENSE = MODE == PK_DENSE;
+    constexpr bool SPLIT = MODE == PK_POOL3;      // staging by the epilogue warps, pooling by PK_POOL_WARPS further warps
     constexpr int EPI_WARPS = pk_epi_warps(DENSE);
     constexpr int MMA_WARP2 = PK_FIRST_EPI + EPI_WARPS;
     pdl_trigger();
@@ -170,6 +177,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     auto res_full = [&](int b) { return ctrl0 + 112u + 8u * b; };   // residual tile landed in staging buffer b
     uint32_t *tmem_slot = (uint32_t *)(ctrl + 104);
     volatile int *abort_flag = (volatile int *)(ctrl + 108);
+    auto sfull = [&](int b) { return ctrl0 + 640u + 8u * b; };      // 3x3-pool kernel: staging buffer b holds a finished group
+    auto sempty = [&](int b) { return ctrl0 + 656u + 8u * b; };     // ... has been pooled and may be overwritten
     auto wfull = [&](int s) { return ctrl0 + 128u + 8u * s; };
     auto wempty = [&](int s) { return ctrl0 + 384u + 8u * s; };
     int2 *lut = (int2 *)(ctrl + 1024);   // entry -> (source slot | tile row << 16, output offset in elements); x < 0: nothing to store
@@ -186,6 +195,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         if (l < p.pstages) { mbar_init(pfull(l), 1); mbar_init(pempty(l), p.MT); }
         if (l < 2) { mbar_init(tfull(l), p.MT); mbar_init(tempty(l), EPI_WARPS); mbar_init(res_full(l), 1); }
         if (l == 2) { mbar_init(epi_bar, EPI_WARPS); *abort_flag = 0; }
+        if (SPLIT && l >= 4 && l < 6) { mbar_init(sfull(l - 4), EPI_WARPS); mbar_init(sempty(l - 4), PK_POOL_WARPS); }
         if (l < p.wstages) { mbar_init(wfull(l), 1); mbar_init(wempty(l), p.MT); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -332,6 +342,81 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             else acc_phase ^= 1u;
         }
         }
+    } else if (SPLIT && warp > MMA_WARP2) {
+        // ------------------------------------------------------------------ 3x3 stride-2 pooling of staged groups
+        // The tile computed conv rows p0 .. p0 + TH - 1 (p0 odd or -1) and holds the windows of (TH - 1) / 2 x (TW - 1) / 2
+        // pooled pixels, all nine slots of each inside the staged tile.  A thread handles up to four (pooled pixel,
+        // 8 filters) items, the same ones in every tile: the shared-memory offsets of their window slots are worked out once.
+        const int ctid = threadIdx.x - (MMA_WARP2 + 1) * 32;
+        constexpr int ITEMS = 512 / (PK_POOL_WARPS * 32);
+        const int groups = (p.FT + 63) / 64;
+        const int tpc = (p.TW - 1) >> 1;
+        const int n_entries = ((p.TH - 1) >> 1) * tpc;
+        const bool clamp_lo = p.act != CPRUNE_ACT_NONE;
+        uint32_t win_off[ITEMS][9];
+        int win_pi[ITEMS], win_pj[ITEMS];
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it) {
+            const int e = ctid + it * (PK_POOL_WARPS * 32);
+            const int ent = e >> 3, chunk = e & 7;
+            win_pi[it] = ent / tpc; win_pj[it] = ent - win_pi[it] * tpc;
+#pragma unroll
+            for (int k = 0; k < 9; ++k) {
+                const int sl = (2 * win_pi[it] + k / 3) * p.Wp + 2 * win_pj[it] + k % 3;
+                win_off[it][k] = (uint32_t)((sl >> 7) * PK_BLOCK_BYTES) + sub_off(sl & 127, chunk);
+            }
+        }
+        uint32_t counter = 0;
+        bool ok = true;
+        // pixels outside the image never win: after ReLU / ReLU6 every value is >= 0 (and every window holds a real
+        // pixel), so they can be replaced by 0 and the maximum taken on the bit patterns; else by -inf
+        const uint4 fill = clamp_lo ? make_uint4(0u, 0u, 0u, 0u) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+        for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+            int tm = item, nt = 0;
+            if (p.tiles_n > 1) { tm = item / p.tiles_n; nt = item - tm * p.tiles_n; }
+            int n, p0, q0;
+            tile_origin(p, tm, n, p0, q0);
+            const int pr0 = (p0 + 1) >> 1, pc0 = (q0 + 1) >> 1;
+            for (int g = 0; g < groups && ok; ++g) {
+                const uint32_t b = counter & 1u;
+                ok = __all_sync(0xffffffffu, mbar_wait(sfull(b), (counter >> 1) & 1u, abort_flag, p.status));
+                if (!ok) break;
+                const uint8_t *buf = smem + (staging0 - base) + b * stage_buf_bytes;
+                const int kg = nt * p.FT + g * 64;
+#pragma unroll
+                for (int it = 0; it < ITEMS; ++it) {
+                    const int e = ctid + it * (PK_POOL_WARPS * 32);
+                    const int chunk = e & 7;
+                    const int pr = pr0 + win_pi[it], pc = pc0 + win_pj[it];
+                    if (e < n_entries * 8 && pr < p.out_h && pc < p.out_w && g * 64 + chunk * 8 < p.FT && kg + chunk * 8 < p.k_pad) {
+                        const int r0 = p0 + 2 * win_pi[it], c0 = q0 + 2 * win_pj[it];
+                        // bit d of a mask: window row / column d lies inside the image
+                        const uint32_t rmask = (r0 >= 0 ? 1u : 0u) | 2u | (r0 + 2 < p.P ? 4u : 0u);
+                        const uint32_t cmask = (c0 >= 0 ? 1u : 0u) | 2u | (c0 + 2 < p.Q ? 4u : 0u);
+                        uint4 w[9];
+#pragma unroll
+                        for (int k = 0; k < 9; ++k) {
+                            const uint4 t = *(const uint4 *)(buf + win_off[it][k]);
+                            w[k] = ((rmask >> (k / 3)) & (cmask >> (k % 3)) & 1u) ? t : fill;
+                        }
+                        uint4 m;
+                        if (clamp_lo) {
+                            const uint4 a0 = bf16x8_max_nonneg(bf16x8_max_nonneg(w[0], w[1]), bf16x8_max_nonneg(w[2], w[3]));
+                            const uint4 a1 = bf16x8_max_nonneg(bf16x8_max_nonneg(w[4], w[5]), bf16x8_max_nonneg(w[6], w[7]));
+                            m = bf16x8_max_nonneg(bf16x8_max_nonneg(a0, a1), w[8]);
+                        } else {
+                            const uint4 a0 = bf16x8_max(bf16x8_max(w[0], w[1]), bf16x8_max(w[2], w[3]));
+                            const uint4 a1 = bf16x8_max(bf16x8_max(w[4], w[5]), bf16x8_max(w[6], w[7]));
+                            m = bf16x8_max(bf16x8_max(a0, a1), w[8]);
+                        }
+                        *(uint4 *)(p.y + (((size_t)n * p.out_h + pr) * p.out_w + pc) * p.k_pad + kg + chunk * 8) = m;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sempty(b));
+                ++counter;
+            }
+        }
     } else {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;
@@ -358,7 +443,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // the shared-memory offsets of their nine window slots are worked out once
         uint32_t win_off[2][9];
         int win_pi[2] = {0, 0}, win_pj[2] = {0, 0};
-        if (!DENSE && p.pool == 2) {
+        if (MODE == PK_GENERAL && p.pool == 2) {
             const int tpc = (p.TW - 1) >> 1;
 #pragma unroll
             for (int it = 0; it < 2; ++it) {
@@ -479,6 +564,11 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 const uint32_t boff = (p.staging_bufs == 2 ? (group_counter & 1u) : 0u) * stage_buf_bytes;
                 uint8_t *buf = smem + (staging0 - base) + boff;
                 const int ch = g * 64 + half * 32;           // this warp's 32 filters of the group
+                if constexpr (SPLIT) {
+                    // the buffer's previous contents (two groups ago) must have been pooled
+                    ok = __all_sync(0xffffffffu, mbar_wait(sempty(group_counter & 1u), ((group_counter >> 1) & 1u) ^ 1u, abort_flag, p.status, false));
+                    if (!ok) break;
+                }
                 if (with_res) {
                     const uint32_t b = p.staging_bufs == 2 ? (group_counter & 1u) : 0u;
                     const uint32_t par = p.staging_bufs == 2 ? ((group_counter >> 1) & 1u) : (group_counter & 1u);
@@ -527,6 +617,13 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                             }
                         }
                     }
+                }
+                if constexpr (SPLIT) {
+                    // hand the staged group to the pooling warps and go on with the next one
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sfull(group_counter & 1u));
+                    ++group_counter;
+                    continue;
                 }
                 if (!p.pool) {
                     // one TMA store per group: the staged slots are TH rows of Wp pixels; the tensor map's box has
@@ -1056,8 +1153,9 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     {
         std::lock_guard<std::mutex> lock(attr_mu);
         if (!attr_set) {
-            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<PK_GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<PK_DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<PK_POOL3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             attr_set = true;
         }
     }
@@ -1088,10 +1186,14 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
     const int grid = total < sms ? total : sms;
+    // a fused 3x3 pool with two staging buffers: the instantiation with separate pooling warps
+    const bool split_pool = p.pool == CPRUNE_POOL_MAX3X3S2 && t.staging_bufs == 2 && !res && !getenv("CPRUNE_PATCH_NO_POOL_WARPS");
     if (t.dense)
-        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<true>, dim3(grid), dim3(PK_THREADS_DENSE), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
+        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<PK_DENSE>, dim3(grid), dim3(pk_threads(PK_DENSE)), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
+    else if (split_pool)
+        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<PK_POOL3>, dim3(grid), dim3(pk_threads(PK_POOL3)), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     else
-        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<false>, dim3(grid), dim3(PK_THREADS), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
+        CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<PK_GENERAL>, dim3(grid), dim3(pk_threads(PK_GENERAL)), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     return CPRUNE_OK;
 }
 
