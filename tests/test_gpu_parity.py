@@ -208,6 +208,16 @@ def test_maxpool_3x3_stride_2(cp, case):
     assert plan.out_h == (P - 1) // 2 + 1
 
 
+def test_maxpool_3x3_stride_2_pooled_by_the_epilogue_warps(cp, monkeypatch):
+    # the fused pool normally runs on separate pooling warps; the measurement switch (read at launch time) selects the
+    # instantiation in which the epilogue warps pool the tile themselves, which plans with one staging buffer use
+    monkeypatch.setenv("CPRUNE_PATCH_NO_POOL_WARPS", "1")
+    check_task(cp, 16, 3, 64, 64, 64, 7, 2, 3, act="relu", pool="max3x3s2", kernel="tensor")
+    check_task(cp, 40, 3, 30, 30, 24, 3, 1, 1, act="none", pool="max3x3s2", kernel="tensor")
+    monkeypatch.delenv("CPRUNE_PATCH_NO_POOL_WARPS")
+    check_task(cp, 40, 3, 30, 30, 24, 3, 1, 1, act="none", pool="max3x3s2", kernel="tensor")
+
+
 @pytest.mark.parametrize("case", [
     # tasks of the benchmarked models at their full batch-64 sizes, i.e. in the launch configuration bench.py times:
     # N, C, H, W, K, R, stride, pad, groups, act, residual, pool
