@@ -158,6 +158,22 @@ def select_indices(w, keep_k: int) -> np.ndarray:
     return kept
 
 
+def select_indices_shared(ws, keep_k: int) -> np.ndarray:
+    """Dependency-aware selection (paper Sec. 3.5, last paragraph): layers whose outputs are added
+    on a shortcut lose the SAME output channels.  The importance of channel k is the sum over the
+    member layers of that channel's L1 norm (each on the 2^-40 grid); the keep_k largest survive,
+    ties keep the lower index.  ws: list of weight tensors that all have K filters."""
+    K = ws[0].shape[0]
+    total = np.zeros(K, dtype=np.int64)
+    for w in ws:
+        assert w.shape[0] == K
+        total += l1_norms(w)
+    assert 1 <= keep_k <= K
+    kept = np.empty(keep_k, dtype=np.int32)
+    _load().oracle_select(_dp(total), K, keep_k, _dp(kept))
+    return kept
+
+
 def select_filters(w, b, keep_k, w_next=None, next_is_depthwise=False):
     """Prune a layer to keep_k filters and make the next layer consistent (paper Sec. 3.5):
     returns (kept, w[kept], b[kept], w_next sliced).  A dense next layer [K2,K,R2,S2] loses
@@ -177,10 +193,22 @@ def select_filters(w, b, keep_k, w_next=None, next_is_depthwise=False):
 
 def prune_model(model: dict, weights: dict):
     """Apply L1 filter pruning to every layer of the table that has a keep count and slice
-    its consumers.  Returns (pruned weights: name -> (w, b), kept: name -> indices)."""
+    its consumers.  Layers that carry the same ``share`` tag write tensors that meet in a
+    residual add: they are ranked together (select_indices_shared) when the first of them is
+    reached and all lose the same filters (the ranking uses the weights as given, before any
+    slicing).  Returns (pruned weights: name -> (w, b), kept:
+    name -> indices)."""
     by = {l["name"]: l for l in model["layers"]}
     out = {k: (w.copy(), b.copy()) for k, (w, b) in weights.items()}
     kept_all = {}
+    # shared groups are ranked once, on the members' weights as given (full width, before any slicing)
+    shared = {}
+    for l in model["layers"]:
+        tag = l.get("share") if l["kind"] == "conv" else None
+        if tag is not None and l["keep"] is not None and tag not in shared:
+            members = [m for m in model["layers"] if m["kind"] == "conv" and m.get("share") == tag]
+            assert all(m["keep"] == l["keep"] for m in members)
+            shared[tag] = select_indices_shared([weights[m["name"]][0] for m in members], l["keep"])
 
     def follow(layer, kept):
         for cname, how in layer["consumers"]:
@@ -196,7 +224,8 @@ def prune_model(model: dict, weights: dict):
     for l in model["layers"]:
         if l["kind"] == "conv" and l["keep"] is not None:
             w, b = out[l["name"]]
-            kept = select_indices(w, l["keep"])
+            tag = l.get("share")
+            kept = select_indices(w, l["keep"]) if tag is None else shared[tag]
             out[l["name"]] = (np.ascontiguousarray(w[kept]), np.ascontiguousarray(b[kept]))
             kept_all[l["name"]] = kept
             follow(l, kept)
@@ -238,6 +267,59 @@ def model_ref(model: dict, weights: dict, x, matched: bool = False, keep_tensors
         else:
             raise ValueError(kind)
     return (t[last], t) if keep_tensors else t[last]
+
+
+# ----------------------------------------------------------------------------
+# pruning decision and task ordering (host-side steps of the method)
+# ----------------------------------------------------------------------------
+
+def prune_step_lcm(L1, L2, unit1: int = 1, unit2: int = 1) -> int:
+    """Minimum number of filters to prune while keeping the structure of a task's program
+    (paper Sec. 3.5, the LCM equation).  L1 and L2 are the factors into which the program splits
+    the two iterators that run over the filters; removing one slice along a factor l of an
+    iterator prunes (product of its factors) / l filters, the smallest such number is
+    product / max factor, and the step that suits both iterators is the least common multiple
+    of the two.  unit1 / unit2: filters behind one count of the factors (1 in the paper's loop
+    nests; larger when the innermost group of filters is fixed by an instruction and cannot
+    shrink)."""
+    def smallest(L, unit):
+        L = [int(v) for v in L]
+        assert L and all(v >= 1 for v in L)
+        prod = 1
+        for v in L:
+            prod *= v
+        return unit * (prod // max(L))
+    a, b = smallest(L1, unit1), smallest(L2, unit2)
+    return a * b // math.gcd(a, b)
+
+
+def task_order(times, counts) -> list:
+    """Tasks ordered by pruning impact = execution time x number of subgraphs that share the
+    task, largest first (paper Sec. 3.3); equal impacts keep the lower index first."""
+    impact = [float(t) * int(c) for t, c in zip(times, counts)]
+    return sorted(range(len(impact)), key=lambda i: (-impact[i], i))
+
+
+def task_table(model: dict) -> list:
+    """The task / subgraph relationship of a layer table (paper Sec. 3.4): conv layers whose
+    shape and fused properties agree form one task.  Returns a list of (key, [layer names]) in
+    order of first appearance; key = (C, K, H, W, R, S, stride, pad, groups, act, residual, pool)
+    with the widths after pruning."""
+    import workloads as wl   # layer tables are data shared with the library's harness
+    m = wl.pruned_shapes(model)
+    sz = wl.spatial_sizes(m)
+    tasks, order = {}, []
+    for l in m["layers"]:
+        if l["kind"] != "conv":
+            continue
+        h, w = sz[l["in"]]
+        key = (l["C"], l["K"], h, w, l["R"], l["S"], l["stride"], l["pad"], l["groups"], l["act"],
+               l.get("res") is not None, l.get("pool"))
+        if key not in tasks:
+            tasks[key] = []
+            order.append(key)
+        tasks[key].append(l["name"])
+    return [(k, tasks[k]) for k in order]
 
 
 def conv_flops(N, C, K, P, Q, R, S, groups=1) -> int:

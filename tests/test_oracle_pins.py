@@ -157,7 +157,7 @@ def test_flop_closed_form_and_paper_totals():
         if line.strip() and not line.startswith("#"):
             name, macs, params = line.split()
             totals[name] = (float(macs), float(params))
-    for name, fn in (("resnet18", wl.resnet18), ("mobilenet_v2", wl.mobilenet_v2)):
+    for name, fn in (("resnet18", wl.resnet18), ("mobilenet_v2", wl.mobilenet_v2), ("mnasnet1_0", wl.mnasnet1_0)):
         got = oracle.model_counts(fn(None))
         assert abs(got["macs"] - totals[name][0]) <= 0.006 * totals[name][0], (name, got)
         assert abs(got["params"] - totals[name][1]) <= 0.01 * totals[name][1], (name, got)
@@ -295,7 +295,8 @@ def test_layer_tables_match_the_pruned_widths():
     assert len(wl.sweep_shapes()) >= 40
 
 
-@pytest.mark.parametrize("name,hw", [("vgg16_cifar", 32), ("resnet18", 32), ("mobilenet_v2", 32)])
+@pytest.mark.parametrize("name,hw", [("vgg16_cifar", 32), ("resnet18", 32), ("mobilenet_v2", 32), ("mnasnet1_0", 32),
+                                     ("resnet18_shared", 32)])
 def test_keep_all_pruning_equals_unpruned_model(name, hw):
     model = _tiny(wl.MODELS[name](), hw)
     weights = wl.model_weights(model)
@@ -312,7 +313,8 @@ def test_keep_all_pruning_equals_unpruned_model(name, hw):
     assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("name,hw", [("vgg16_cifar", 32), ("resnet18", 32), ("mobilenet_v2", 32)])
+@pytest.mark.parametrize("name,hw", [("vgg16_cifar", 32), ("resnet18", 32), ("mobilenet_v2", 32), ("mnasnet1_0", 32),
+                                     ("resnet18_shared", 32)])
 def test_pruned_model_equals_unpruned_with_dropped_filters_zeroed(name, hw):
     model = _tiny(wl.MODELS[name](), hw)
     weights = wl.model_weights(model)
@@ -353,3 +355,185 @@ def test_generator_is_counter_based_and_normal():
     assert not np.array_equal(wl.normal(5, 4, 1000), a)
     z = wl.normal(9, 0, 400000)
     assert abs(z.mean()) < 0.01 and abs(z.std() - 1) < 0.01 and abs(np.mean(z ** 4) - 3) < 0.1
+
+
+# ------------------------------------------------------------------ shared (dependency-aware) selection
+
+def test_shared_selection_hand_made():
+    # two member layers, four channels.  Per-channel norms: layer A = 1, 5, 2, 4; layer B = 6, 1, 2, 2.
+    # Summed: 7, 6, 4, 6 -> keep 2: channels 0 and 1 (the tie between 1 and 3 keeps the lower index);
+    # keep 3: 0, 1, 3.  Ranking either layer alone would choose differently (A alone: 1 and 3).
+    a = np.zeros((4, 1, 1, 1), dtype=np.float32)
+    b = np.zeros((4, 2, 1, 1), dtype=np.float32)
+    a[:, 0, 0, 0] = [1, -5, 2, 4]
+    b[:, 0, 0, 0] = [6, 0.5, -2, 1]
+    b[:, 1, 0, 0] = [0, -0.5, 0, 1]
+    assert oracle.select_indices_shared([a, b], 2).tolist() == [0, 1]
+    assert oracle.select_indices_shared([a, b], 3).tolist() == [0, 1, 3]
+    assert oracle.select_indices(a, 2).tolist() == [1, 3]
+    # one member: the plain selection; member order does not matter
+    w = wl.normal_f32(41, 1, (23, 5, 3, 3), 0.1)
+    v = wl.normal_f32(41, 2, (23, 7, 1, 1), 0.1)
+    for keep in (1, 9, 23):
+        assert np.array_equal(oracle.select_indices_shared([w], keep), oracle.select_indices(w, keep))
+        assert np.array_equal(oracle.select_indices_shared([w, v], keep), oracle.select_indices_shared([v, w], keep))
+    # the group norm is the norm of the members' filters laid side by side
+    both = np.concatenate([w.reshape(23, -1), v.reshape(23, -1)], axis=1).reshape(23, -1, 1, 1)
+    assert np.array_equal(oracle.select_indices_shared([w, v], 11), oracle.select_indices(both, 11))
+
+
+def test_shared_groups_of_the_resnet_table_keep_the_same_filters():
+    model = _tiny(wl.resnet18_shared(), 32)
+    weights = wl.model_weights(model)
+    pw, kept = oracle.prune_model(model, weights)
+    for stage, members in ((1, ["stem", "l1b1_conv2", "l1b2_conv2"]), (3, ["l3b1_down", "l3b1_conv2", "l3b2_conv2"])):
+        ref = oracle.select_indices_shared([weights[m][0] for m in members], (3 * [64, 128, 256, 512][stage - 1]) // 4)
+        for m in members:
+            assert np.array_equal(kept[m], ref), m
+    assert pw["fc"][0].shape == (1000, 384) and pw["l2b1_down"][0].shape == (96, 48, 1, 1)
+
+
+# ------------------------------------------------------------------ pruning decision, task ordering, task table
+
+def _paper_examples():
+    ex = {}
+    for line in open(os.path.join(GOLDEN, "paper_worked_examples.txt")):
+        if line.strip() and not line.startswith("#"):
+            key, val = line.split(":", 1)
+            ex[key.strip()] = val.strip()
+    return ex
+
+
+def test_prune_step_matches_the_papers_worked_examples():
+    ex = _paper_examples()
+    for key in ("lcm_fast_program", "lcm_slow_program"):
+        l1, l2, want = ex[key].split("|")
+        L1 = [int(v) for v in l1.split("x")]
+        L2 = [int(v) for v in l2.split("x")]
+        assert oracle.prune_step_lcm(L1, L2) == int(want), key
+    # the smallest slice of 4 x 8 x 16 filters is 512 / 16; of 3 x 5 it is 3; lcm(32, 3) = 96
+    assert oracle.prune_step_lcm([4, 8, 16], [3, 5]) == 96
+    assert oracle.prune_step_lcm([7], [7]) == 1               # one unsplit iterator: any single filter
+    assert oracle.prune_step_lcm([2, 6], [2, 6], 16, 8) == 32   # 16 * 12 / 6 = 32 and 8 * 12 / 6 = 16
+
+
+def test_task_order_matches_the_papers_worked_example():
+    ex = _paper_examples()
+    times = [float(v) for v in ex["order_times"].split()]
+    counts = [int(v) for v in ex["order_subgraphs"].split()]
+    impacts = [float(v) for v in ex["order_impacts"].split()]
+    assert [round(t * c, 3) for t, c in zip(times, counts)] == impacts
+    assert [i + 1 for i in oracle.task_order(times, counts)] == [int(v) for v in ex["order_result"].split()]
+    assert oracle.task_order([1.0, 2.0, 1.0, 0.5], [2, 1, 2, 4]) == [0, 1, 2, 3]     # all impacts equal: index order
+    assert oracle.task_order([], []) == []
+
+
+def test_task_table_groups_identical_shapes():
+    # pruned ResNet-18: 20 conv layers, 15 distinct tasks; pruned MobileNetV2: 52 conv layers, 30 distinct
+    for fn, layers, tasks in ((wl.resnet18, 20, 15), (wl.mobilenet_v2, 52, 30)):
+        tab = oracle.task_table(fn())
+        assert sum(len(names) for _, names in tab) == layers and len(tab) == tasks
+    tab = dict((tuple(n), k) for k, n in oracle.task_table(wl.resnet18()))
+    assert ("l1b1_conv1", "l1b2_conv1") in tab and ("l3b1_conv2", "l3b2_conv2") in tab
+
+
+# ------------------------------------------------------------------ wiring of the layer tables
+# The networks written out a second time, straight from their published architecture, with
+# torch.nn.functional in float64 and none of the tables' wiring (tensor names, residual sources,
+# activation placement): only the weights are looked up, by layer name.
+
+def _t(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).double()
+
+
+def _fconv(x, wb, stride=1, pad=0, groups=1, act=None):
+    import torch.nn.functional as F
+    y = F.conv2d(x, _t(wb[0]), _t(wb[1]), stride=stride, padding=pad, groups=groups)
+    if act == "relu":
+        y = F.relu(y)
+    elif act == "relu6":
+        y = torch.clamp(y, 0.0, 6.0)
+    return y
+
+
+def _torch_vgg16(W, x):
+    import torch.nn.functional as F
+    i = 0
+    for block in (2, 2, 3, 3, 3):
+        for _ in range(block):
+            i += 1
+            x = _fconv(x, W["c%d" % i], 1, 1, act="relu")
+        x = F.max_pool2d(x, 2, 2)
+    x = x.flatten(1)
+    x = F.relu(F.linear(x, _t(W["fc1"][0]), _t(W["fc1"][1])))
+    return F.linear(x, _t(W["fc2"][0]), _t(W["fc2"][1]))
+
+
+def _torch_resnet18(W, x):
+    import torch.nn.functional as F
+    x = _fconv(x, W["stem"], 2, 3, act="relu")
+    x = F.max_pool2d(x, 3, 2, 1)
+    for stage in (1, 2, 3, 4):
+        for block in (1, 2):
+            pre = "l%db%d" % (stage, block)
+            stride = 2 if (stage > 1 and block == 1) else 1
+            shortcut = _fconv(x, W[pre + "_down"], stride, 0) if (pre + "_down") in W else x
+            h = _fconv(x, W[pre + "_conv1"], stride, 1, act="relu")
+            h = _fconv(h, W[pre + "_conv2"], 1, 1)
+            x = F.relu(h + shortcut)
+    x = x.mean(dim=(2, 3))
+    return F.linear(x, _t(W["fc"][0]), _t(W["fc"][1]))
+
+
+def _torch_inverted_residuals(W, x, settings, act, first_block):
+    b = first_block
+    for expand, cout, repeats, stride, k in settings:
+        for j in range(repeats):
+            s = stride if j == 0 else 1
+            pre = "b%d" % b
+            h = x
+            if (pre + "_exp") in W:
+                h = _fconv(h, W[pre + "_exp"], act=act)
+            ch = h.shape[1]
+            h = _fconv(h, W[pre + "_dw"], s, k // 2, groups=ch, act=act)
+            h = _fconv(h, W[pre + "_proj"])
+            x = x + h if (s == 1 and x.shape[1] == cout) else h
+            b += 1
+    return x
+
+
+def _torch_mobilenet_v2(W, x):
+    import torch.nn.functional as F
+    x = _fconv(x, W["stem"], 2, 1, act="relu6")
+    settings = [(1, 16, 1, 1, 3), (6, 24, 2, 2, 3), (6, 32, 3, 2, 3), (6, 64, 4, 2, 3), (6, 96, 3, 1, 3),
+                (6, 160, 3, 2, 3), (6, 320, 1, 1, 3)]
+    x = _torch_inverted_residuals(W, x, settings, "relu6", 1)
+    x = _fconv(x, W["last"], act="relu6").mean(dim=(2, 3))
+    return F.linear(x, _t(W["fc"][0]), _t(W["fc"][1]))
+
+
+def _torch_mnasnet(W, x):
+    import torch.nn.functional as F
+    x = _fconv(x, W["stem"], 2, 1, act="relu")
+    x = _fconv(x, W["sep_dw"], 1, 1, groups=32, act="relu")
+    x = _fconv(x, W["sep_pw"])
+    settings = [(3, 24, 3, 2, 3), (3, 40, 3, 2, 5), (6, 80, 3, 2, 5), (6, 96, 2, 1, 3), (6, 192, 4, 2, 5), (6, 320, 1, 1, 3)]
+    x = _torch_inverted_residuals(W, x, settings, "relu", 1)
+    x = _fconv(x, W["last"], act="relu").mean(dim=(2, 3))
+    return F.linear(x, _t(W["fc"][0]), _t(W["fc"][1]))
+
+
+@pytest.mark.parametrize("name,forward,hw", [("vgg16_cifar", _torch_vgg16, 32), ("resnet18", _torch_resnet18, 32),
+                                             ("mobilenet_v2", _torch_mobilenet_v2, 32), ("mnasnet1_0", _torch_mnasnet, 32),
+                                             ("resnet18", _torch_resnet18, 64)])
+def test_table_wiring_against_the_architecture_written_out(name, forward, hw):
+    for pruned in (False, True):
+        model = _tiny(wl.MODELS[name](), hw)
+        weights = wl.model_weights(model)
+        if pruned:
+            weights, _ = oracle.prune_model(model, weights)
+        x = wl.model_input(model, 2)
+        ref = forward(weights, _t(x).permute(0, 3, 1, 2)).numpy()
+        got = oracle.model_ref(model, weights, x)
+        assert got.shape == ref.shape
+        assert np.max(np.abs(got - ref)) <= 1e-10 * np.max(np.abs(ref)), (name, pruned)

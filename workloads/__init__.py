@@ -21,6 +21,8 @@ Layer tables.  A model is a dict ``{"name", "input": (H, W, C), "layers": [...],
              optional ``res`` (tensor added before the activation), optional
              ``pool`` = "max2x2" (2x2 stride-2 max-pool applied to the result),
              ``keep`` = filters kept by L1 pruning (None: layer is not pruned),
+             optional ``share`` = tag of a group of layers whose outputs meet in a residual
+             add and therefore keep the SAME filters (one ranking for the whole group),
              ``consumers`` = layers whose input channels follow this layer's
              kept filters: list of (layer name, how) with how in
              {"in_channels", "depthwise", "fc_in"}.
@@ -82,10 +84,10 @@ def normal_f32(seed: int, stream: int, shape, std: float = 1.0) -> np.ndarray:
 # ----------------------------------------------------------------------------
 
 def _conv(name, tin, tout, C, K, R, stride, pad, act, groups=1, res=None, pool=None,
-          keep=None, consumers=()):
+          keep=None, consumers=(), share=None):
     return {"kind": "conv", "name": name, "in": tin, "out": tout, "C": C, "K": K, "R": R, "S": R,
             "stride": stride, "pad": pad, "groups": groups, "act": act, "res": res, "pool": pool,
-            "keep": keep, "consumers": list(consumers)}
+            "keep": keep, "consumers": list(consumers), "share": share}
 
 
 def single_task() -> dict:
@@ -118,30 +120,56 @@ def vgg16_cifar(keep=VGG16_KEEP) -> dict:
     return {"name": "vgg16_cifar", "input": (32, 32, 3), "layers": layers, "output": "logits", "seed": 1002}
 
 
-def resnet18(keep_num=7, keep_den=10) -> dict:
+def resnet18(keep_num=7, keep_den=10, out_num=None, out_den=4) -> dict:
     """ResNet-18 for 3x224x224 inputs.  The first conv of every BasicBlock keeps
-    floor(keep_num * width / keep_den) filters; block outputs keep their width so that
-    the residual adds keep their shapes.  keep_num=None gives the unpruned network."""
-    layers = [_conv("stem", "x", "s0", 3, 64, 7, 2, 3, "relu"),
+    floor(keep_num * width / keep_den) filters.  With out_num=None block outputs keep their
+    width so that the residual adds keep their shapes; keep_num=None gives the unpruned network.
+    With out_num set, the tensors that meet in the residual adds of a stage (the stem or the
+    stage's 1x1 shortcut conv, and the second conv of both blocks) are pruned too, to
+    floor(out_num * width / out_den) filters, and all of them lose the same filters (one
+    ``share`` group per stage: the dependency-aware pruning of the paper's Sec. 3.5)."""
+    def okeep(w):
+        return None if out_num is None else (out_num * w) // out_den
+
+    # consumers of a stage's shared tensors are filled in as the readers appear
+    layers = [_conv("stem", "x", "s0", 3, 64, 7, 2, 3, "relu", keep=okeep(64), share="stage1" if out_num else None),
               {"kind": "maxpool", "name": "pool0", "in": "s0", "out": "p0", "k": 3, "stride": 2, "pad": 1}]
     t, c = "p0", 64
+    writer = layers[0]          # the layer that wrote tensor t
     for si, w in enumerate([64, 128, 256, 512], start=1):
+        tag = "stage%d" % si if out_num else None
         for bi in (1, 2):
             stride = 2 if (si > 1 and bi == 1) else 1
             pre = "l%db%d" % (si, bi)
             keep = None if keep_num is None else (keep_num * w) // keep_den
             ident = t
             if stride != 1 or c != w:
-                layers.append(_conv(pre + "_down", t, pre + "_id", c, w, 1, stride, 0, "none"))
+                layers.append(_conv(pre + "_down", t, pre + "_id", c, w, 1, stride, 0, "none", keep=okeep(w), share=tag))
                 ident = pre + "_id"
+                if out_num:
+                    writer["consumers"].append((pre + "_down", "in_channels"))
+            if out_num:
+                writer["consumers"].append((pre + "_conv1", "in_channels"))
             layers.append(_conv(pre + "_conv1", t, pre + "_h", c, w, 3, stride, 1, "relu", keep=keep,
                                 consumers=[(pre + "_conv2", "in_channels")]))
-            layers.append(_conv(pre + "_conv2", pre + "_h", pre + "_o", w, w, 3, 1, 1, "relu", res=ident))
+            layers.append(_conv(pre + "_conv2", pre + "_h", pre + "_o", w, w, 3, 1, 1, "relu", res=ident,
+                                keep=okeep(w), share=tag))
+            writer = layers[-1]
             t, c = pre + "_o", w
     layers.append({"kind": "gap", "name": "gap", "in": t, "out": "g"})
     layers.append({"kind": "fc", "name": "fc", "in": "g", "out": "logits", "in_features": 512,
                    "out_features": 1000, "act": "none"})
+    if out_num:
+        writer["consumers"].append(("fc", "fc_in"))
     return {"name": "resnet18", "input": (224, 224, 3), "layers": layers, "output": "logits", "seed": 1003}
+
+
+def resnet18_shared() -> dict:
+    """Pruned ResNet-18 whose block outputs are pruned as well, to 3/4 of their width, with one
+    shared filter set per stage (see resnet18)."""
+    m = resnet18(out_num=3)
+    m["name"] = "resnet18_shared"
+    return m
 
 
 _MBV2_SETTING = [(1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2), (6, 96, 3, 1),
@@ -180,8 +208,45 @@ def mobilenet_v2(keep_num=3, keep_den=4) -> dict:
     return {"name": "mobilenet_v2", "input": (224, 224, 3), "layers": layers, "output": "logits", "seed": 1004}
 
 
+# MnasNet-B1, depth multiplier 1.0 (Tan et al. 2019, the "MnasNet1.0" of the paper's Sec. 4.1):
+# (expansion, output channels, repeats, stride of the first block, depthwise kernel size)
+_MNASNET_SETTING = [(3, 24, 3, 2, 3), (3, 40, 3, 2, 5), (6, 80, 3, 2, 5), (6, 96, 2, 1, 3),
+                    (6, 192, 4, 2, 5), (6, 320, 1, 1, 3)]
+
+
+def mnasnet1_0(keep_num=3, keep_den=4) -> dict:
+    """MnasNet1.0 for 3x224x224 inputs: 3x3 stride-2 stem to 32 channels, a depthwise-separable
+    block to 16, six stacks of inverted-residual blocks (1x1 expand + ReLU, 3x3 or 5x5 depthwise
+    + ReLU, 1x1 project, residual add where the block keeps its shape), 1x1 conv to 1280, global
+    average pool, FC 1280 -> 1000.  Every expand layer keeps floor(keep_num * width / keep_den)
+    filters; its depthwise layer and the project layer's inputs follow."""
+    layers = [_conv("stem", "x", "s0", 3, 32, 3, 2, 1, "relu"),
+              _conv("sep_dw", "s0", "s1", 32, 32, 3, 1, 1, "relu", groups=32),
+              _conv("sep_pw", "s1", "s2", 32, 16, 1, 1, 0, "none")]
+    t, c, bi = "s2", 16, 0
+    for tfac, cout, n, s, k in _MNASNET_SETTING:
+        for j in range(n):
+            bi += 1
+            stride = s if j == 0 else 1
+            pre = "b%d" % bi
+            hidden = c * tfac
+            keep = None if keep_num is None else (keep_num * hidden) // keep_den
+            layers.append(_conv(pre + "_exp", t, pre + "_e", c, hidden, 1, 1, 0, "relu", keep=keep,
+                                consumers=[(pre + "_dw", "depthwise")]))
+            layers.append(_conv(pre + "_dw", pre + "_e", pre + "_d", hidden, hidden, k, stride, k // 2, "relu",
+                                groups=hidden, consumers=[(pre + "_proj", "in_channels")]))
+            res = t if (stride == 1 and c == cout) else None
+            layers.append(_conv(pre + "_proj", pre + "_d", pre + "_o", hidden, cout, 1, 1, 0, "none", res=res))
+            t, c = pre + "_o", cout
+    layers.append(_conv("last", t, "l0", 320, 1280, 1, 1, 0, "relu"))
+    layers.append({"kind": "gap", "name": "gap", "in": "l0", "out": "g"})
+    layers.append({"kind": "fc", "name": "fc", "in": "g", "out": "logits", "in_features": 1280,
+                   "out_features": 1000, "act": "none"})
+    return {"name": "mnasnet1_0", "input": (224, 224, 3), "layers": layers, "output": "logits", "seed": 1005}
+
+
 MODELS = {"single_task": single_task, "vgg16_cifar": vgg16_cifar, "resnet18": resnet18,
-          "mobilenet_v2": mobilenet_v2}
+          "mobilenet_v2": mobilenet_v2, "mnasnet1_0": mnasnet1_0, "resnet18_shared": resnet18_shared}
 
 
 def layer_by_name(model: dict) -> dict:
