@@ -47,6 +47,11 @@ enum { CPRUNE_ACT_NONE = 0, CPRUNE_ACT_RELU = 1, CPRUNE_ACT_RELU6 = 2 };
 enum { CPRUNE_POOL_NONE = 0, CPRUNE_POOL_MAX2X2 = 1, CPRUNE_POOL_MAX3X3S2 = 2 };
 /* kernel families a plan can choose */
 enum { CPRUNE_KERNEL_AUTO = 0, CPRUNE_KERNEL_DIRECT = 1, CPRUNE_KERNEL_TENSOR = 2, CPRUNE_KERNEL_DEPTHWISE = 3 };
+/* option flags of a plan (bits of cprune_task_opts.flags; part of the plan's cache key).  They select between
+ * implementations that compute the same values, for tests and measurements:
+ *   IM2COL_ONLY             tensor family: never the kernel that keeps the input patch in shared memory
+ *   POOL_ON_EPILOGUE_WARPS  fused 3x3 stride-2 pool: pooled by the epilogue warps instead of separate pooling warps */
+enum { CPRUNE_FLAG_IM2COL_ONLY = 1, CPRUNE_FLAG_POOL_ON_EPILOGUE_WARPS = 2, CPRUNE_FLAG_ALL = 3 };
 
 typedef struct cprune_plan cprune_plan;
 typedef struct cprune_model cprune_model;
@@ -109,6 +114,16 @@ cprune_status cprune_select_filters_static(const float *w, const float *b, int K
                                            int32_t *kept_idx, float *w_out, float *b_out, float *w_next_out,
                                            void *stream);
 
+/* Dependency-aware selection (paper Sec. 3.5, last paragraph: layers whose outputs meet in a shortcut add
+ * lose the same output channels).  The importance of filter index k is the sum, over the n_members layers,
+ * of that layer's grid norm of filter k; the keep_k largest are kept, ties keep the lower index.
+ *   w_list   HOST array of n_members device pointers, member m is float32 [K][inner[m]]
+ *   inner    HOST array: weights per filter of each member (C*R*S), each <= 2^13
+ *   kept_idx device, int32 [keep_k], ascending; slice the members and their consumers with the gather calls
+ * Workspace as for cprune_select_filters.  With one member the result equals cprune_select_filters'. */
+cprune_status cprune_select_shared(const float *const *w_list, const size_t *inner, int n_members, int K, int keep_k,
+                                   int32_t *kept_idx, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Row gather out[j][:] = in[idx[j]][:] (inner floats per row) and column gather
  * out[o][j][:] = in[o][idx[j]][:] for further consumers of the same kept_idx (a depthwise layer's
  * bias, the project layer behind a depthwise layer, the first FC layer).  All pointers device. */
@@ -126,6 +141,7 @@ typedef struct {
     int residual;     /* 1: a residual tensor [N][P][Q][k_pad] is added before the activation */
     int pool;         /* CPRUNE_POOL_*: max-pool applied to the activated result */
     int kernel;       /* CPRUNE_KERNEL_AUTO or a forced family (for tests and measurements) */
+    int flags;        /* CPRUNE_FLAG_* bits, 0 by default */
 } cprune_task_opts;
 
 typedef struct {
@@ -145,6 +161,13 @@ typedef struct {
                                  of a tile stays in shared memory and every tap reads it (stride-1 tasks, stems),
                                  2 = as 1, for 1x1 tasks whose output tile is one contiguous range of y: staged as it
                                  lies in memory and stored by a single bulk copy */
+    int splits;               /* slices of the reduction that go to different CTAs (1: no split); > 1 adds a second launch */
+    /* How the program splits the two iterators that run over the filters (paper Sec. 3.5): the compute iterator
+     * (filter tiles x instruction-sized groups per tile) and the store iterator (filter tiles x 16-byte pieces per
+     * tile); each count stands for `unit` filters that one instruction or one store handles and that cannot shrink. */
+    int split_compute[2], unit_compute;
+    int split_store[2], unit_store;
+    double est_us;            /* the planner's own estimate of the task's time (its cost model, microseconds) */
 } cprune_plan_info;
 
 /* Host only; launches nothing.  opts == NULL means bias + ReLU, no residual, no pool, AUTO.
@@ -162,6 +185,23 @@ cprune_status cprune_plan_release(cprune_plan *plan);
 cprune_status cprune_cache_clear(int *n_left);
 /* Number of distinct plans in the cache and number of lookups that hit (host, either may be NULL). */
 cprune_status cprune_cache_stats(int *n_plans, long long *n_hits);
+
+/* ---------------------------------------------------------------------------------------------
+ * Pruning decision (paper Sec. 3.5): how many filters to prune from a task so that the pruned task keeps
+ * the structure of its program.  The paper takes, for each of the two iterators over the filters, the
+ * smallest slice of its split (product of the factors / largest factor) and prunes the least common
+ * multiple of the two.  Here the program is the plan: *step = LCM(unit_compute * prod(split_compute) /
+ * max(split_compute), unit_store * prod(split_store) / max(split_store)).  Host only.
+ * cprune_task_estimate gives the planner's estimate of the same task with k_new filters (all else equal;
+ * it plans that task, which the cache then holds), so that a caller can ask which filter count makes the
+ * task a step faster before it prunes anything.  Errors: INVALID_ARG (null, k_new < 1), UNSUPPORTED. */
+cprune_status cprune_prune_step(const cprune_plan *plan, int *step /* host */);
+cprune_status cprune_task_estimate(const cprune_plan *plan, int k_new, double *est_us /* host */);
+
+/* Task ordering (paper Sec. 3.3): order[0..n) receives the task indices sorted by pruning impact =
+ * execution time x number of subgraphs that share the task, largest first; equal impacts keep the lower
+ * index first.  Host arrays. */
+cprune_status cprune_task_order(const double *times, const int *counts, int n, int *order);
 
 /* One-time layout change of a (pruned) layer's parameters for its plan:
  * w float32 [K][C/groups][R][S] -> bfloat16 (round to nearest even) [k_alloc][R][S][c_pad] with zero
@@ -235,11 +275,31 @@ cprune_status cprune_model_tensor(const cprune_model *model, int id, const void 
 cprune_status cprune_model_copy_tensor(const cprune_model *model, int id, void *dst, void *stream);
 /* Kernel launches one cprune_model_run enqueues. */
 int cprune_model_launches(const cprune_model *model);
+
+/* The model's task table (paper Sec. 3.4: which subgraphs share which task): one entry per distinct plan among
+ * the model's conv tasks, in order of first appearance.  entries (host) receives at most max_entries entries;
+ * *n_entries the number of distinct tasks. */
+typedef struct {
+    const cprune_plan *plan;   /* the shared task */
+    int count;                 /* subgraphs (conv tasks of the model) that use it */
+    int first_task;            /* index into the model's task list of the first of them */
+} cprune_task_entry;
+cprune_status cprune_model_task_table(const cprune_model *model, cprune_task_entry *entries, int max_entries, int *n_entries);
+/* Times every entry of the task table on the device: the entry's first subgraph is run `reps` times back to back
+ * on the model's own buffers between two CUDA events (after one untimed run); ms (host, one value per table entry)
+ * receives the mean milliseconds per run.  Blocks until the measurements are done.  Feed ms and the counts to
+ * cprune_task_order to get the paper's pruning priority. */
+cprune_status cprune_model_time_tasks(cprune_model *model, int reps, double *ms, void *stream);
 cprune_status cprune_model_destroy(cprune_model *model);
 
 /* Reads and clears the device status word after synchronising `stream` (this call blocks).
  * Returns CPRUNE_OK, CPRUNE_ERR_TIMEOUT or CPRUNE_ERR_BAD_DATA. */
 cprune_status cprune_poll_device_status(void *stream);
+/* Self-test of the bounded waits: launches one small CTA that waits, with a limit of 65,536 cycles, on a
+ * barrier that nothing will ever signal (the same wait routine the tensor-core kernels use with their one-second
+ * limit).  The wait gives up, raises the time-out bit of the device status word and the kernel returns; the next
+ * cprune_poll_device_status therefore reports CPRUNE_ERR_TIMEOUT once, and the device stays usable. */
+cprune_status cprune_selftest_wait_timeout(void *stream);
 
 #ifdef __cplusplus
 }

@@ -18,6 +18,7 @@ ACT = {"none": 0, "relu": 1, "relu6": 2}
 POOL = {None: 0, "none": 0, "max2x2": 1, "max3x3s2": 2}
 KERNEL = {"auto": 0, "direct": 1, "tensor": 2, "depthwise": 3}
 KERNEL_NAMES = {v: k for k, v in KERNEL.items()}
+FLAGS = {"im2col_only": 1, "pool_on_epilogue_warps": 2}
 OP_CONV, OP_MAXPOOL, OP_GAP, OP_FC = 1, 2, 3, 4
 
 # every symbol include/cprune.h declares
@@ -27,7 +28,9 @@ EXPORTS = [
     "cprune_plan_release", "cprune_cache_clear", "cprune_cache_stats", "cprune_pack_weights", "cprune_task_run",
     "cprune_cast_input", "cprune_widen_output", "cprune_maxpool", "cprune_global_avgpool", "cprune_fc_pack",
     "cprune_fc", "cprune_model_create", "cprune_model_run", "cprune_model_run_host", "cprune_model_tensor", "cprune_model_copy_tensor", "cprune_model_launches",
-    "cprune_model_destroy", "cprune_poll_device_status",
+    "cprune_model_destroy", "cprune_poll_device_status", "cprune_select_shared", "cprune_prune_step",
+    "cprune_task_estimate", "cprune_task_order", "cprune_model_task_table", "cprune_model_time_tasks",
+    "cprune_selftest_wait_timeout",
 ]
 
 
@@ -38,7 +41,7 @@ class CpruneError(RuntimeError):
 
 
 class TaskOpts(ctypes.Structure):
-    _fields_ = [("activation", c_int), ("residual", c_int), ("pool", c_int), ("kernel", c_int)]
+    _fields_ = [("activation", c_int), ("residual", c_int), ("pool", c_int), ("kernel", c_int), ("flags", c_int)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -46,10 +49,18 @@ class PlanInfo(ctypes.Structure):
                                       "out_w", "c_pad", "k_pad", "kernel", "tile_m", "tile_n", "tile_k", "stages",
                                       "tiles_m", "tiles_n", "k_alloc")] + \
                [("packed_weight_bytes", c_size_t), ("packed_bias_bytes", c_size_t), ("workspace_bytes", c_size_t),
-                ("flops", c_double), ("algorithmic_bytes", c_double), ("padded_flops", c_double), ("variant", c_int)]
+                ("flops", c_double), ("algorithmic_bytes", c_double), ("padded_flops", c_double), ("variant", c_int),
+                ("splits", c_int), ("split_compute", c_int * 2), ("unit_compute", c_int), ("split_store", c_int * 2),
+                ("unit_store", c_int), ("est_us", c_double)]
 
     def as_dict(self):
-        return {n: getattr(self, n) for n, _ in self._fields_}
+        d = {n: getattr(self, n) for n, _ in self._fields_}
+        d["split_compute"], d["split_store"] = list(d["split_compute"]), list(d["split_store"])
+        return d
+
+
+class TaskEntry(ctypes.Structure):
+    _fields_ = [("plan", c_void_p), ("count", c_int), ("first_task", c_int)]
 
 
 class TaskDesc(ctypes.Structure):
@@ -100,6 +111,14 @@ def lib():
         L.cprune_model_launches.argtypes = [c_void_p]
         L.cprune_model_destroy.argtypes = [c_void_p]
         L.cprune_poll_device_status.argtypes = [c_void_p]
+        L.cprune_select_shared.argtypes = [POINTER(c_void_p), POINTER(c_size_t), c_int, c_int, c_int, c_void_p, c_void_p,
+                                           c_size_t, c_void_p]
+        L.cprune_prune_step.argtypes = [c_void_p, POINTER(c_int)]
+        L.cprune_task_estimate.argtypes = [c_void_p, c_int, POINTER(c_double)]
+        L.cprune_task_order.argtypes = [POINTER(c_double), POINTER(c_int), c_int, POINTER(c_int)]
+        L.cprune_model_task_table.argtypes = [c_void_p, POINTER(TaskEntry), c_int, POINTER(c_int)]
+        L.cprune_model_time_tasks.argtypes = [c_void_p, c_int, POINTER(c_double), c_void_p]
+        L.cprune_selftest_wait_timeout.argtypes = [c_void_p]
         _lib = L
     return _lib
 
@@ -185,6 +204,21 @@ def cprune_select_filters_static(w, keep_k, kept_idx, w_out, b=None, b_out=None,
     return kept_idx, w_out, b_out, w_next_out
 
 
+def cprune_select_shared(ws, keep_k, workspace=None, stream=None):
+    """ws: list of float32 device tensors that all have K filters (dim 0).  Returns kept_idx int32 [keep_k]: the
+    filters with the largest norm summed over the members."""
+    ws = [_dev_f32(w) for w in ws]
+    K = ws[0].shape[0]
+    ptrs = (c_void_p * len(ws))(*[w.data_ptr() for w in ws])
+    inner = (c_size_t * len(ws))(*[w.numel() // K for w in ws])
+    kept = torch.empty(max(int(keep_k), 0), dtype=torch.int32, device=ws[0].device)
+    if workspace is None:
+        workspace = torch.empty(max(cprune_select_workspace_bytes(K), 16), dtype=torch.uint8, device=ws[0].device)
+    _check(lib().cprune_select_shared(ptrs, inner, len(ws), K, int(keep_k), _ptr(kept), _ptr(workspace),
+                                      workspace.numel(), _stream(stream)), "cprune_select_shared")
+    return kept
+
+
 def cprune_gather_rows(t, idx, stream=None):
     """out[j] = t[idx[j]] along dim 0."""
     t = _dev_f32(t)
@@ -231,11 +265,36 @@ class Plan:
 
 
 def cprune_task_plan(N, C, H, W, K, R, S, stride, pad, groups=1, activation="relu", residual=False, pool=None,
-                     kernel="auto") -> Plan:
-    opts = TaskOpts(ACT[activation], 1 if residual else 0, POOL[pool], KERNEL[kernel])
+                     kernel="auto", flags=()) -> Plan:
+    fl = 0
+    for f in flags:
+        fl |= FLAGS[f]
+    opts = TaskOpts(ACT[activation], 1 if residual else 0, POOL[pool], KERNEL[kernel], fl)
     h = c_void_p()
     _check(lib().cprune_task_plan(N, C, H, W, K, R, S, stride, pad, groups, byref(opts), byref(h)), "cprune_task_plan")
     return Plan(h)
+
+
+def cprune_prune_step(plan: Plan) -> int:
+    step = c_int()
+    _check(lib().cprune_prune_step(plan.handle, byref(step)), "cprune_prune_step")
+    return step.value
+
+
+def cprune_task_estimate(plan: Plan, k_new: int) -> float:
+    us = c_double()
+    _check(lib().cprune_task_estimate(plan.handle, int(k_new), byref(us)), "cprune_task_estimate")
+    return us.value
+
+
+def cprune_task_order(times, counts):
+    n = len(times)
+    assert len(counts) == n
+    t = (c_double * max(n, 1))(*[float(v) for v in times])
+    c = (c_int * max(n, 1))(*[int(v) for v in counts])
+    o = (c_int * max(n, 1))()
+    _check(lib().cprune_task_order(t, c, n, o), "cprune_task_order")
+    return [o[j] for j in range(n)]
 
 
 def cprune_cache_stats():
@@ -346,6 +405,21 @@ class Model:
         _check(lib().cprune_model_copy_tensor(self.handle, tid, _ptr(out), _stream(stream)), "cprune_model_copy_tensor")
         return out
 
+    def task_table(self):
+        """[(plan handle value, count, first task index)] of the model's distinct conv tasks."""
+        n = c_int()
+        _check(lib().cprune_model_task_table(self.handle, None, 0, byref(n)), "cprune_model_task_table")
+        arr = (TaskEntry * max(n.value, 1))()
+        _check(lib().cprune_model_task_table(self.handle, arr, n.value, byref(n)), "cprune_model_task_table")
+        return [(arr[j].plan, arr[j].count, arr[j].first_task) for j in range(n.value)]
+
+    def time_tasks(self, reps=5, stream=None):
+        """Milliseconds per run of every entry of the task table (blocks)."""
+        n = len(self.task_table())
+        ms = (c_double * max(n, 1))()
+        _check(lib().cprune_model_time_tasks(self.handle, int(reps), ms, _stream(stream)), "cprune_model_time_tasks")
+        return [ms[j] for j in range(n)]
+
     def __del__(self):
         try:
             if self.handle and _lib is not None:
@@ -385,6 +459,10 @@ def cprune_model_run_host(model: Model, x_host, logits_host, stream=None):
 
 def cprune_poll_device_status(stream=None):
     _check(lib().cprune_poll_device_status(_stream(stream)), "cprune_poll_device_status")
+
+
+def cprune_selftest_wait_timeout(stream=None):
+    _check(lib().cprune_selftest_wait_timeout(_stream(stream)), "cprune_selftest_wait_timeout")
 
 
 __all__ = [n for n in dir() if n.startswith("cprune_")] + ["Plan", "Model", "TaskDesc", "CpruneError", "lib",

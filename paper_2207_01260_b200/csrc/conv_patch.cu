@@ -22,10 +22,10 @@
 //                stay resident in shared memory for the whole kernel;
 //   warps 3, 12  tcgen05.mma issue, one warp per accumulator block;
 //   warps 4..11  epilogue: tcgen05.ld, bias (+ residual), activation, bf16 into a swizzled staging
-//                buffer, then all 256 threads copy the valid pixels out with 16-byte stores, eight
-//                threads per pixel (whole 128-byte lines; stores of 16 bytes per thread at a pixel
-//                stride were measured to be several times slower); a 2x2 max-pool is taken while
-//                copying.
+//                buffer, then ONE TMA store per group of 64 filters whose box is the tile's rows x
+//                Wp pixels (wrap-around columns, rows below the image and filters beyond k_pad lie
+//                outside the tensor map and are not written).  With a fused max-pool the staged
+//                tile is pooled and copied out by hand instead, eight threads per output pixel.
 // Every wait is bounded (see sm100_ptx.cuh); on expiry the CTA raises STATUS_TIMEOUT and leaves.
 #include <cuda.h>
 
@@ -576,7 +576,6 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     if (!ok) break;
                 }
                 for (int mb = 0; mb < p.MT; ++mb) {
-                    const int slot = mb * 128 + trow;
                     uint32_t v[32];
 #pragma unroll
                     for (int sb = 0; sb < 2; ++sb)
@@ -819,7 +818,6 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     plan->pre_bytes = 0;
     PatchGeometry g;
     if (!patch_geometry(i, &g)) return CPRUNE_ERR_UNSUPPORTED;
-    const int Wp = g.Wp;
     const bool pool = plan->opts.pool == CPRUNE_POOL_MAX2X2;
     const bool pool3 = plan->opts.pool == CPRUNE_POOL_MAX3X3S2;
     if (pool && (plan->opts.residual || (i.P & 1) || (i.Q & 1))) return CPRUNE_ERR_UNSUPPORTED;
@@ -831,10 +829,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     const int RS = g.kR * g.kS;
     double best = 1e30;
     PatchTiling bt = {};
-    const char *force_mt = getenv("CPRUNE_PATCH_MT");       // measurement overrides
-    const char *force_tn = getenv("CPRUNE_PATCH_TN");
     for (int MT = 1; MT <= 2; ++MT) {
-        if (force_mt && atoi(force_mt) != MT) continue;
       // candidate tile shapes: whole-width rows; for the 3x3 pool (2 tpr + 1) x (2 tpc + 1) conv pixels around tpr x tpc pooled ones
       const int n_shapes = pool3 ? 32 * 32 : 1;
       for (int shape = 0; shape < n_shapes; ++shape) {
@@ -861,7 +856,6 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             tiles_per_img = (i.P + TH - 1) / TH;
         }
         for (int tiles_n = 1; tiles_n <= 8; ++tiles_n) {
-            if (force_tn && atoi(force_tn) != tiles_n) continue;
             // with several filter tiles every tile ends on a 64-filter boundary: the stores are 64 filters wide and
             // only the tensor's own edge clips them
             const int FT = round_up((k16 + tiles_n - 1) / tiles_n, tiles_n > 1 ? 64 : 16);
@@ -876,10 +870,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             // tiles long, so the ring is as deep as fits)
             int ps_max = 2;
             if (cblks > 2 && patch_bytes <= 32 * 1024) ps_max = cblks < PK_MAX_PATCH_STAGES ? cblks : PK_MAX_PATCH_STAGES;
-            const char *force_ps = getenv("CPRUNE_PATCH_PSTAGES");      // measurement override
-            if (g.flat) ps_max = force_ps ? atoi(force_ps) : PK_MAX_PATCH_STAGES;
-            if (ps_max < 2) ps_max = 2;
-            if (ps_max > PK_MAX_PATCH_STAGES) ps_max = PK_MAX_PATCH_STAGES;
+            if (g.flat) ps_max = PK_MAX_PATCH_STAGES;
           for (int pstages = ps_max; pstages >= 2; --pstages) {
             const int fixed = 1024 + pstages * patch_bytes + PK_CTRL_BYTES;
             const int budget = 227 * 1024 - fixed;
@@ -888,17 +879,15 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             // flat tasks with one filter tile stage the tile as it lies in memory (k_pad filters per pixel) when that fits
             // and the pixel pitch is an odd number of 16-byte pieces (no bank conflicts between neighbouring pixels;
             // 32-byte pixels conflict two-way and still gain, measured)
-            const char *force_dense = getenv("CPRUNE_PATCH_DENSE");     // measurement override: 0 = never
             const int dense_bytes = round_up(128 * MT * i.k_pad * 2, 1024);
-            const int dense = g.flat && tiles_n == 1 && (((i.k_pad >> 3) & 1) || i.k_pad == 16) && dense_bytes <= 40 * 1024 && !(force_dense && force_dense[0] == '0');
+            const int dense = g.flat && tiles_n == 1 && (((i.k_pad >> 3) & 1) || i.k_pad == 16) && dense_bytes <= 40 * 1024;
             const int stage_bytes = dense ? dense_bytes : MT * PK_BLOCK_BYTES;
             int staging_bufs = sb_max, wstages = 0, resident = 0;
             // resident filters when the whole set of this filter tile fits
             // (with a residual, only beside two staging buffers: with one buffer the residual of a group can only be
             // fetched after the previous group's store has drained, which costs more than streaming the filters)
-            const char *force_res = getenv("CPRUNE_PATCH_RESIDENT");      // measurement override: 0 = never, 1 = whenever it fits
-            const int sb_res_min = (plan->opts.residual && !(force_res && force_res[0] == '1')) ? 2 : sb_min;
-            if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES && !(force_res && force_res[0] == '0')) {
+            const int sb_res_min = plan->opts.residual ? 2 : sb_min;
+            if (tiles_n == 1 && RS * cblks <= PK_MAX_WSTAGES) {
                 for (int sb = sb_max; sb >= sb_res_min && !resident; --sb)
                     if (RS * cblks * w_stage + sb * stage_bytes <= budget) { resident = 1; staging_bufs = sb; wstages = RS * cblks; }
             }
@@ -954,6 +943,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
     i.padded_flops = 2.0 * (double)i.tiles_m * i.tile_m * (double)i.k_alloc * RS * ksteps * 16.0;
     plan->smem_bytes = 1024 + bt.pstages * bt.patch_bytes + bt.wstages * round_up(bt.FT * RB, 1024) +
                        bt.staging_bufs * bt.stage_bytes + PK_CTRL_BYTES;
+    plan->est_us = best / 1900.0 + 4.0;      // cycles at about 1.9 GHz plus launch, set-up and drain
     return CPRUNE_OK;
 }
 
@@ -1148,15 +1138,19 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
         std::memcpy(&tm_y, &plan->tm_y, sizeof(CUtensorMap));
         std::memcpy(&tm_res, res ? &plan->tm_res : &plan->tm_y, sizeof(CUtensorMap));
     }
+    // the shared-memory limit of a kernel is a per-device attribute
     static std::mutex attr_mu;
-    static bool attr_set = false;
+    static bool attr_set[64] = {false};
     {
+        int dev = 0;
+        CPRUNE_CUDA_CHECK(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return CPRUNE_ERR_UNSUPPORTED;
         std::lock_guard<std::mutex> lock(attr_mu);
-        if (!attr_set) {
+        if (!attr_set[dev]) {
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<PK_GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<PK_DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_patch_kernel<PK_POOL3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            attr_set = true;
+            attr_set[dev] = true;
         }
     }
     PatchParams p;
@@ -1187,7 +1181,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
     const int grid = total < sms ? total : sms;
     // a fused 3x3 pool with two staging buffers: the instantiation with separate pooling warps
-    const bool split_pool = p.pool == CPRUNE_POOL_MAX3X3S2 && t.staging_bufs == 2 && !res && !getenv("CPRUNE_PATCH_NO_POOL_WARPS");
+    const bool split_pool = p.pool == CPRUNE_POOL_MAX3X3S2 && t.staging_bufs == 2 && !res && !(plan->opts.flags & CPRUNE_FLAG_POOL_ON_EPILOGUE_WARPS);
     if (t.dense)
         CPRUNE_CUDA_CHECK(launch_chained(conv_patch_kernel<PK_DENSE>, dim3(grid), dim3(pk_threads(PK_DENSE)), (size_t)plan->smem_bytes, st, tm_x, tm_w, tm_y, tm_res, p));
     else if (split_pool)

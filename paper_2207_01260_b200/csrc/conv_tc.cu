@@ -4,17 +4,16 @@
 //   D[pixel][k] = sum over (r, s, c) of  X[pixel shifted by tap (r,s)][c] * Wt[k][r][s][c]
 //   GEMM-M = N*P*Q output pixels,  GEMM-N = K filters,  GEMM-K = R*S*C
 //
-// One persistent CTA per SM, N_PRODUCERS + 9 warps, three roles (warp numbers for N_PRODUCERS = 4; measured: one
-// producer warp is enough for this kernel, which is bound by shared-memory bandwidth):
-//   warps 0..3  producers: per (tap, 64-channel block) one im2col-mode TMA load of PT pixels x 64
+// One persistent CTA per SM, 10 warps, three roles (measured: one producer warp is enough for this
+// kernel, which is bound by shared-memory bandwidth):
+//   warp 0      producer: per (tap, 64-channel block) one im2col-mode TMA load of PT pixels x 64
 //               channels of the activation tensor (zero fill for the padding border and for
 //               channels beyond c_pad) and one tiled TMA load of FT filters x 64 channels, both
-//               into 128-byte-swizzled shared memory, completion on an mbarrier; the producer warps
-//               take the pipeline stages in turn;
-//   warp 4      one elected lane issues tcgen05.mma (K = 16 per instruction, bf16 x bf16 ->
+//               into 128-byte-swizzled shared memory, completion on an mbarrier;
+//   warp 1      one elected lane issues tcgen05.mma (K = 16 per instruction, bf16 x bf16 ->
 //               float32) with the accumulator in tensor memory; two accumulator buffers so
 //               that the epilogue of one tile overlaps the main loop of the next;
-//   warps 5..12 epilogue: tcgen05.ld the accumulator, bias (+ residual), activation, bf16,
+//   warps 2..9  epilogue: tcgen05.ld the accumulator, bias (+ residual), activation, bf16,
 //               write 64-filter-wide sub-tiles into swizzled shared memory, TMA-store them to
 //               the NHWC output (the store clips rows beyond the last pixel and filters beyond
 //               k_pad by itself).
@@ -725,17 +724,18 @@ __global__ void __launch_bounds__(256) splitk_finalize_kernel(const float *__res
     if (valid && sub == 0) y[e] = pack8(f);
 }
 
-// 128 x 128 identity in bf16: the filter-side operand of the residual blocks (see the producer).
-static __device__ __align__(256) __nv_bfloat16 g_identity[128 * 128];
+// 128 x 128 identity in bf16 (1.0 = 0x3F80): the filter-side operand of the residual blocks (see the producer).
+// Initialised in the library image, so no launch and no synchronisation is needed before its first use.
+struct IdentityBits {
+    uint16_t v[128 * 128];
+    constexpr IdentityBits() : v{} {
+        for (int i = 0; i < 128; ++i) v[i * 128 + i] = 0x3F80;
+    }
+};
+static __device__ __align__(256) const IdentityBits g_identity = IdentityBits();
 
-__global__ void fill_identity_kernel() {
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < 128 * 128) g_identity[i] = __float2bfloat16_rn((i / 128 == i % 128) ? 1.f : 0.f);
-}
-
-// Device address of the identity matrix on the current device; filled on first use (one small
-// launch on the given stream, ordered before the conv kernel that follows it there).
-static cprune_status identity_address(void **out, cudaStream_t st) {
+// Device address of the identity matrix on the current device (looked up once per device).
+static cprune_status identity_address(void **out) {
     static std::mutex mu;
     static void *ptrs[64] = {nullptr};
     int dev = 0;
@@ -745,9 +745,6 @@ static cprune_status identity_address(void **out, cudaStream_t st) {
     if (!ptrs[dev]) {
         void *p = nullptr;
         CPRUNE_CUDA_CHECK(cudaGetSymbolAddress(&p, g_identity));
-        fill_identity_kernel<<<64, 256, 0, st>>>();
-        CPRUNE_LAUNCH_CHECK("fill_identity_kernel");
-        CPRUNE_CUDA_CHECK(cudaStreamSynchronize(st));   // later launches may come from other streams
         ptrs[dev] = p;
     }
     *out = ptrs[dev];
@@ -797,8 +794,7 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     if (i.groups != 1) return CPRUNE_ERR_UNSUPPORTED;
     // stride-1 tasks with more than one tap: patch kernel when its tile is well filled
     plan->patch = 0;
-    const char *no_patch = getenv("CPRUNE_NO_PATCH");      // measurement override
-    if (!(no_patch && no_patch[0] == '1') && plan_conv_patch(plan) == CPRUNE_OK) return CPRUNE_OK;
+    if (!(plan->opts.flags & CPRUNE_FLAG_IM2COL_ONLY) && plan_conv_patch(plan) == CPRUNE_OK) return CPRUNE_OK;
     if (i.R > 16 || i.S > 16 || i.pad > 64 || i.stride > 8) return CPRUNE_ERR_UNSUPPORTED;
     if (i.W > 65535 || i.H > 65535) return CPRUNE_ERR_UNSUPPORTED;
     const long long M = (long long)i.N * i.P * i.Q;
@@ -808,9 +804,6 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     // stride-2 stems with odd pad and odd S: read the image as pixel pairs (16 channels per pair), which halves
     // the number of loads and doubles their row width; the packed filters get one zero tap in front of each row
     if (plan->small_c && i.stride == 2 && (i.W & 1) == 0 && (i.pad & 1) == 1 && (i.S & 1) == 1) plan->small_c = 2;
-    if (const char *e = getenv("CPRUNE_STEM_PAIRS")) {      // measurement override
-        if (e[0] == '0' && plan->small_c == 2) plan->small_c = 1;
-    }
     plan->s_packed = plan->small_c == 2 ? i.S + 1 : i.S;
     // Orientation.  K <= 128: filters on the 128-row side (256 pixels per MMA) -- except for tasks with one or two
     // K blocks and at most 32 filters (MobileNetV2 project layers), where the pixel-major epilogue, in which every
@@ -834,10 +827,6 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
             if (ft_next < 128) break;
             if ((long long)tiles_m * tiles_n >= 148) break;
             tiles_n = next;
-        }
-        if (const char *e = getenv("CPRUNE_TC_TILES_N")) {     // measurement override
-            const int v = atoi(e);
-            if (v >= (k16 + 255) / 256 && v <= 16) tiles_n = v;
         }
         // with several filter tiles every tile must end on a 64-filter boundary: the staged stores
         // are 64 filters wide and only the tensor's own edge clips them
@@ -882,10 +871,6 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
             if (t < best * 0.9) { best = t; plan->splits = sp; }
         }
     }
-    if (const char *force = getenv("CPRUNE_FORCE_SPLITS")) {   // measurement override
-        int sp = atoi(force);
-        if (sp >= 1 && !plan->small_c && sp <= iters && (sp - 1) * ((iters + sp - 1) / sp) < iters) plan->splits = sp;
-    }
     // A 2x2 max-pool is fused when a tile holds whole pairs of image rows: Q a power of two with the
     // four pixels of a window in one warp (pixel-major: Q <= 16) or in one thread's 64-pixel group
     // (filter-major: Q <= 32).  The split-K finalize kernel pools for any even P, Q.
@@ -897,6 +882,16 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     }
     plan->ipp = (iters + plan->splits - 1) / plan->splits;
     plan->partial_bytes = plan->splits > 1 ? (size_t)plan->splits * (size_t)M * i.k_alloc * 4 : 0;
+    {
+        // estimate: per K block the tensor pipe needs 4 MMAs of N / 2 cycles, shared memory takes the TMA writes of
+        // both operands and the MMAs' operand reads at 128 bytes per clock; about 1.9 GHz; launch and drain on top
+        const int mma_n = plan->orient == ORIENT_PIX ? FT : PT;
+        const double tensor = 4.0 * mma_n / 2.0;
+        const double smem = (PT + FT) * 128.0 / 128.0 + 4.0 * (128.0 + mma_n) * 32.0 / 128.0;
+        const double per_block = tensor > smem ? tensor : smem;
+        const double waves = (double)ceil_div(tiles * plan->splits, 148);
+        plan->est_us = waves * (plan->ipp * per_block + 2000.0) / 1900.0 + 4.0 + (plan->splits > 1 ? 3.0 : 0.0);
+    }
     return CPRUNE_OK;
 }
 
@@ -975,7 +970,7 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled(res)");
         void *ident = nullptr;
-        cprune_status s2 = identity_address(&ident, stream);
+        cprune_status s2 = identity_address(&ident);
         if (s2 != CPRUNE_OK) return s2;
         cuuint64_t idims[2] = {128, 128};
         cuuint64_t istrides[1] = {256};
@@ -1021,15 +1016,18 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
         std::memcpy(&tm_id, mma_res ? &plan->tm_id : &plan->tm_y, sizeof(CUtensorMap));
     }
     static std::mutex attr_mu;
-    static int attr_set = 0;
+    static int attr_set[64] = {0};     // the shared-memory limit of a kernel is a per-device attribute
     {
+        int dev = 0;
+        CPRUNE_CUDA_CHECK(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return CPRUNE_ERR_UNSUPPORTED;
         std::lock_guard<std::mutex> lock(attr_mu);
-        if (!attr_set) {
+        if (!attr_set[dev]) {
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_PIX, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_PIX, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_FILT, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(conv_tc_kernel<ORIENT_FILT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-            attr_set = 1;
+            attr_set[dev] = 1;
         }
     }
     TcParams p;

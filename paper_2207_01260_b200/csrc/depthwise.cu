@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
 // Tile of output pixels per CTA and channel groups per CTA.
 // Channel groups (of 8 channels) per CTA: between 4 and 9, whichever wastes the fewest lanes in
 // the last channel block (c_pad/8 = 18 -> 9, 14 -> 7, 4 -> 4); larger wins ties.
-static int dw_groups(int c8) {
+int depthwise_groups(int c8) {
     if (c8 <= 9) return c8;
     int best = 8;
     double best_util = 0.0;
@@ -183,7 +183,7 @@ static int dw_groups(int c8) {
 // Tile of output pixels per CTA and channel groups per CTA.
 static void dw_tile(const cprune_plan_info &i, int *TH, int *TW, int *G) {
     const int c8 = i.c_pad / 8;
-    *G = dw_groups(c8);
+    *G = depthwise_groups(c8);
     int tw = 112 / *G;                      // about 112 threads per CTA: small patches, several CTAs per SM
     if (i.stride == 2 && tw > 28) tw = 28;  // keeps the input patch small
     *TW = i.Q < tw ? i.Q : tw;
@@ -229,13 +229,16 @@ cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, 
     if (blocks > 0x7fffffffLL || p.IW > 256 || p.IH > 256) return CPRUNE_ERR_UNSUPPORTED;
     const int smem = p.IH * p.IW * p.G * 16;
     static std::mutex attr_mu;
-    static int attr_set = 0;
+    static int attr_set[64] = {0};     // the shared-memory limit of a kernel is a per-device attribute
     {
+        int dev = 0;
+        CPRUNE_CUDA_CHECK(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return CPRUNE_ERR_UNSUPPORTED;
         std::lock_guard<std::mutex> lock(attr_mu);
-        if (!attr_set) {
+        if (!attr_set[dev]) {
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(depthwise3x3_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
             CPRUNE_CUDA_CHECK(cudaFuncSetAttribute(depthwise3x3_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-            attr_set = 1;
+            attr_set[dev] = 1;
         }
     }
     if (smem > 100 * 1024) return CPRUNE_ERR_UNSUPPORTED;

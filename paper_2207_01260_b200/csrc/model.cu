@@ -281,6 +281,53 @@ cprune_status cprune_model_copy_tensor(const cprune_model *m, int id, void *dst,
 
 int cprune_model_launches(const cprune_model *m) { return m ? m->launches : 0; }
 
+cprune_status cprune_model_task_table(const cprune_model *m, cprune_task_entry *entries, int max_entries, int *n_entries) {
+    if (!m || !n_entries || max_entries < 0 || (max_entries > 0 && !entries)) return CPRUNE_ERR_INVALID_ARG;
+    std::vector<cprune_task_entry> table;
+    for (size_t t = 0; t < m->tasks.size(); ++t) {
+        const cprune_task_desc &d = m->tasks[t];
+        if (d.op != CPRUNE_OP_CONV) continue;
+        bool found = false;
+        for (auto &e : table)
+            if (e.plan == d.plan) { ++e.count; found = true; break; }
+        if (!found) table.push_back(cprune_task_entry{d.plan, 1, (int)t});
+    }
+    *n_entries = (int)table.size();
+    for (int j = 0; j < (int)table.size() && j < max_entries; ++j) entries[j] = table[j];
+    return CPRUNE_OK;
+}
+
+cprune_status cprune_model_time_tasks(cprune_model *m, int reps, double *ms, void *stream) {
+    if (!m || !ms || reps < 1) return CPRUNE_ERR_INVALID_ARG;
+    int n = 0;
+    cprune_status s = cprune_model_task_table(m, nullptr, 0, &n);
+    if (s != CPRUNE_OK) return s;
+    std::vector<cprune_task_entry> table(n);
+    s = cprune_model_task_table(m, table.data(), n, &n);
+    if (s != CPRUNE_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    CPRUNE_CUDA_CHECK(cudaEventCreate(&e0));
+    CPRUNE_CUDA_CHECK(cudaEventCreate(&e1));
+    for (int j = 0; j < n && s == CPRUNE_OK; ++j) {
+        const cprune_task_desc &d = m->tasks[table[j].first_task];
+        void *pin = tensor_ptr(m, d.in), *pout = tensor_ptr(m, d.out);
+        const void *res = d.res >= 0 ? tensor_ptr(m, d.res) : nullptr;
+        for (int r = 0; r <= reps && s == CPRUNE_OK; ++r) {
+            if (r == 1 && cudaEventRecord(e0, st) != cudaSuccess) s = CPRUNE_ERR_CUDA;   // run 0 is the untimed one
+            if (s == CPRUNE_OK) s = task_run_internal(d.plan, pin, d.w, d.b, res, pout, m->workspace, st, false);
+        }
+        if (s != CPRUNE_OK) break;
+        float t = 0.f;
+        if (cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+            cudaEventElapsedTime(&t, e0, e1) != cudaSuccess) { s = cuda_fail(cudaGetLastError(), "task timing"); break; }
+        ms[j] = (double)t / reps;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return s;
+}
+
 cprune_status cprune_model_destroy(cprune_model *m) {
     if (!m) return CPRUNE_ERR_INVALID_ARG;
     for (auto &g : m->graphs)

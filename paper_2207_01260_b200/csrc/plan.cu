@@ -13,12 +13,9 @@ namespace cprune {
 
 static thread_local bool g_chain_launch = false;
 bool chain_launch_enabled() { return g_chain_launch; }
-void set_chain_launch(bool on) {
-    const char *off = getenv("CPRUNE_NO_PDL");     // measurement override
-    g_chain_launch = on && !(off && off[0] == '1');
-}
+void set_chain_launch(bool on) { g_chain_launch = on; }
 
-using PlanKey = std::array<int, 14>;
+using PlanKey = std::array<int, 15>;
 
 struct PlanCache {
     std::mutex mu;
@@ -38,6 +35,7 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     i.N = key[0]; i.C = key[1]; i.H = key[2]; i.W = key[3]; i.K = key[4]; i.R = key[5]; i.S = key[6];
     i.stride = key[7]; i.pad = key[8]; i.groups = key[9];
     pl->opts.activation = key[10]; pl->opts.residual = key[11]; pl->opts.pool = key[12]; pl->opts.kernel = key[13];
+    pl->opts.flags = key[14];
     pl->refs = 0;
     i.P = (i.H + 2 * i.pad - i.R) / i.stride + 1;
     i.Q = (i.W + 2 * i.pad - i.S) / i.stride + 1;
@@ -77,8 +75,36 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     }
     if (st != CPRUNE_OK) { delete pl; return st; }
     i.kernel = family;
-    i.variant = (family == CPRUNE_KERNEL_TENSOR && pl->patch) ? (pl->pt.dense ? 2 : 1) : 0;
     const double rs = (double)i.R * i.S;
+    i.algorithmic_bytes = 2.0 * ((double)i.N * i.H * i.W * i.C + (double)i.N * i.out_h * i.out_w * i.K +
+                                 (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
+                                 (double)i.K * (i.C / i.groups) * rs) + 4.0 * i.K;
+    // how the program splits the filter axis (see cprune_prune_step)
+    i.splits = family == CPRUNE_KERNEL_TENSOR ? pl->splits : 1;
+    if (family == CPRUNE_KERNEL_TENSOR && (pl->patch || pl->orient == 0)) {
+        // filters on the MMA's column side: tiles_n tiles of tile_n filters, built from 16-filter instruction groups
+        // (64-filter groups when there are several tiles: tiles end on store-box boundaries), stored in 16-byte pieces
+        i.unit_compute = i.tiles_n > 1 ? 64 : 16;
+        i.split_compute[0] = i.tiles_n; i.split_compute[1] = i.tile_n / i.unit_compute;
+        i.unit_store = 8;
+        i.split_store[0] = i.tiles_n; i.split_store[1] = i.tile_n / 8;
+    } else if (family == CPRUNE_KERNEL_DEPTHWISE) {
+        // channel blocks (CTAs along the channels) x channel groups of 8 per CTA
+        const int c8 = i.c_pad / 8;
+        const int g = depthwise_groups(c8);
+        i.unit_compute = i.unit_store = 8;
+        i.split_compute[0] = i.split_store[0] = (c8 + g - 1) / g;
+        i.split_compute[1] = i.split_store[1] = g;
+        pl->est_us = i.algorithmic_bytes / 3.0e6 + 4.0;
+    } else {
+        // filters on the 128-row side of the MMA (any count up to 128 costs the same) or one thread per 8 filters:
+        // the filter axis is only cut into the 8-filter pieces of the memory layout
+        i.unit_compute = i.unit_store = 8;
+        i.split_compute[0] = i.split_store[0] = 1;
+        i.split_compute[1] = i.split_store[1] = i.k_pad / 8;
+        if (family == CPRUNE_KERNEL_DIRECT) pl->est_us = i.flops / 15.0e6 + 4.0;
+    }
+    i.variant = (family == CPRUNE_KERNEL_TENSOR && pl->patch) ? (pl->pt.dense ? 2 : 1) : 0;
     const int s_packed = (family == CPRUNE_KERNEL_TENSOR && pl->s_packed > 0) ? pl->s_packed : i.S;
     i.packed_weight_bytes = depthwise ? (size_t)(rs * i.c_pad * 2) : (size_t)i.k_alloc * i.R * s_packed * i.c_pad * 2;
     if (family == CPRUNE_KERNEL_TENSOR && pl->patch && pl->narrow) i.packed_weight_bytes = packed_weight_bytes_patch(pl);
@@ -88,9 +114,7 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     pl->pool_bytes = separate_pool ? ((size_t)i.N * i.P * i.Q * i.k_pad * 2 + 255) / 256 * 256 : 0;
     // (patch kernel on a regrouped stem: the regrouped input takes the place of the partial sums)
     i.workspace_bytes = pl->pool_bytes + (family == CPRUNE_KERNEL_TENSOR ? pl->partial_bytes + pl->pre_bytes : 0);
-    i.algorithmic_bytes = 2.0 * ((double)i.N * i.H * i.W * i.C + (double)i.N * i.out_h * i.out_w * i.K +
-                                 (pl->opts.residual ? (double)i.N * i.P * i.Q * i.K : 0.0) +
-                                 (double)i.K * (i.C / i.groups) * rs) + 4.0 * i.K;
+    i.est_us = pl->est_us;
     *out = pl;
     return CPRUNE_OK;
 }
@@ -135,10 +159,10 @@ cprune_status cprune_task_plan(int N, int C, int H, int W, int K, int R, int S, 
     if (N <= 0 || C <= 0 || H <= 0 || W <= 0 || K <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0 || groups <= 0)
         return CPRUNE_ERR_INVALID_ARG;
     if (H + 2 * pad < R || W + 2 * pad < S) return CPRUNE_ERR_INVALID_ARG;
-    cprune_task_opts o = {CPRUNE_ACT_RELU, 0, CPRUNE_POOL_NONE, CPRUNE_KERNEL_AUTO};
+    cprune_task_opts o = {CPRUNE_ACT_RELU, 0, CPRUNE_POOL_NONE, CPRUNE_KERNEL_AUTO, 0};
     if (opts) o = *opts;
     if (o.activation < 0 || o.activation > 2 || o.pool < 0 || o.pool > 2 || o.kernel < 0 || o.kernel > 3 ||
-        (o.residual != 0 && o.residual != 1))
+        (o.residual != 0 && o.residual != 1) || (o.flags & ~CPRUNE_FLAG_ALL))
         return CPRUNE_ERR_INVALID_ARG;
     if (groups != 1) {
         if (groups != C || K != C) return CPRUNE_ERR_UNSUPPORTED;
@@ -147,7 +171,7 @@ cprune_status cprune_task_plan(int N, int C, int H, int W, int K, int R, int S, 
     int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
     if (o.pool == CPRUNE_POOL_MAX2X2 && ((P & 1) || (Q & 1))) return CPRUNE_ERR_INVALID_ARG;
     if ((long long)N * P * Q > 0x7fffffffLL || (long long)N * H * W > 0x7fffffffLL) return CPRUNE_ERR_UNSUPPORTED;
-    PlanKey key = {N, C, H, W, K, R, S, stride, pad, groups, o.activation, o.residual, o.pool, o.kernel};
+    PlanKey key = {N, C, H, W, K, R, S, stride, pad, groups, o.activation, o.residual, o.pool, o.kernel, o.flags};
     PlanCache &c = cache();
     std::lock_guard<std::mutex> lock(c.mu);
     auto it = c.plans.find(key);

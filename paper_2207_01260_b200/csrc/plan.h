@@ -49,6 +49,7 @@ struct cprune_plan {
     int narrow = 0;                 // patch kernel on a regrouped 16-channel input (stems with few channels)
     size_t pre_bytes = 0;           // regrouped input in the workspace
     PatchTiling pt = {};
+    double est_us = 0.0;            // the planner's cost-model estimate of the task's time
 };
 
 namespace cprune {
@@ -59,6 +60,8 @@ cprune_status launch_conv_direct(const cprune_plan *plan, const void *x, const v
 // depthwise 3x3
 cprune_status launch_depthwise(cprune_plan *plan, const void *x, const void *w, const float *b,
                                const void *res, void *y, cudaStream_t st);
+// channel groups (of 8 channels) one depthwise CTA handles, for c8 groups in the tensor
+int depthwise_groups(int c8);
 // tcgen05 implicit GEMM
 cprune_status plan_conv_tensor(cprune_plan *plan);  // fills tile fields of plan->info; UNSUPPORTED if not eligible
 cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w, const float *b, const void *res,

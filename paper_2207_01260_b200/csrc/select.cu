@@ -38,8 +38,9 @@ int *device_status_word() {
 
 constexpr int NORM_THREADS = 256;
 
+// accumulate != 0: the norm is added to what norms[] holds (integer adds: any order gives the same bits)
 __global__ void __launch_bounds__(NORM_THREADS) l1_norm_kernel(const float *__restrict__ w, size_t inner,
-                                                                long long *__restrict__ norms, int *status) {
+                                                                long long *__restrict__ norms, int *status, int accumulate) {
     const float *row = w + (size_t)blockIdx.x * inner;
     long long acc = 0;
     bool bad = false;
@@ -56,7 +57,7 @@ __global__ void __launch_bounds__(NORM_THREADS) l1_norm_kernel(const float *__re
     if (threadIdx.x == 0) {
         long long s = 0;
         for (int i = 0; i < NORM_THREADS / 32; ++i) s += part[i];
-        norms[blockIdx.x] = s;
+        norms[blockIdx.x] = accumulate ? norms[blockIdx.x] + s : s;
     }
 }
 
@@ -170,7 +171,7 @@ cprune_status select_launch(const float *w, const float *b, int K, int C, int R,
                             float *w_out, float *b_out, float *w_next_out, long long *norms, int *keep,
                             int *status, cudaStream_t st) {
     size_t inner = (size_t)C * R * S;
-    l1_norm_kernel<<<K, NORM_THREADS, 0, st>>>(w, inner, norms, status);
+    l1_norm_kernel<<<K, NORM_THREADS, 0, st>>>(w, inner, norms, status, 0);
     CPRUNE_LAUNCH_CHECK("l1_norm_kernel");
     rank_kernel<<<(K + RANK_THREADS - 1) / RANK_THREADS, RANK_THREADS, 0, st>>>(norms, K, keep_k, keep);
     CPRUNE_LAUNCH_CHECK("rank_kernel");
@@ -264,6 +265,33 @@ cprune_status cprune_select_filters_static(const float *w, const float *b, int K
     int *keep = (int *)(scratch + STATIC_NORM_BYTES);
     return select_launch(w, b, K, C, R, S, keep_k, w_next, K2, R2, S2, next_is_depthwise, kept_idx, w_out, b_out,
                          w_next_out, norms, keep, status, (cudaStream_t)stream);
+}
+
+cprune_status cprune_select_shared(const float *const *w_list, const size_t *inner, int n_members, int K, int keep_k,
+                                   int32_t *kept_idx, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!w_list || !inner || n_members < 1 || K <= 0 || !kept_idx) return CPRUNE_ERR_INVALID_ARG;
+    if (keep_k < 1 || keep_k > K) return CPRUNE_ERR_INVALID_ARG;
+    for (int m = 0; m < n_members; ++m) {
+        if (!w_list[m] || inner[m] == 0) return CPRUNE_ERR_INVALID_ARG;
+        if (inner[m] > 8192) return CPRUNE_ERR_UNSUPPORTED;
+    }
+    if ((size_t)n_members > (size_t)1 << 9) return CPRUNE_ERR_UNSUPPORTED;   // keeps the int64 sums far from overflow
+    if (!workspace || ((uintptr_t)workspace & 15)) return CPRUNE_ERR_INVALID_ARG;
+    if (workspace_bytes < cprune_select_workspace_bytes(K)) return CPRUNE_ERR_WORKSPACE_TOO_SMALL;
+    int *status = device_status_word();
+    if (!status) return cuda_fail(cudaGetLastError(), "status word");
+    cudaStream_t st = (cudaStream_t)stream;
+    long long *norms = (long long *)workspace;
+    int *keep = (int *)((char *)workspace + align_up((size_t)K * sizeof(long long), 256));
+    for (int m = 0; m < n_members; ++m) {
+        l1_norm_kernel<<<K, NORM_THREADS, 0, st>>>(w_list[m], inner[m], norms, status, m > 0);
+        CPRUNE_LAUNCH_CHECK("l1_norm_kernel");
+    }
+    rank_kernel<<<(K + RANK_THREADS - 1) / RANK_THREADS, RANK_THREADS, 0, st>>>(norms, K, keep_k, keep);
+    CPRUNE_LAUNCH_CHECK("rank_kernel");
+    compact_kernel<<<1, COMPACT_THREADS, 0, st>>>(keep, K, kept_idx);
+    CPRUNE_LAUNCH_CHECK("compact_kernel");
+    return CPRUNE_OK;
 }
 
 cprune_status cprune_gather_rows(const float *in, int rows, size_t inner, const int32_t *idx, int n_idx, float *out,

@@ -47,14 +47,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 
 // Bounded wait.  Returns false when the limit expired here or (if watch_abort) another role gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
-                                          bool watch_abort = true) {
+                                          bool watch_abort = true, long long limit_cycles = WAIT_LIMIT_CYCLES) {
     for (int i = 0; i < 64; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (watch_abort && *abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit_cycles) {
             atomicOr(status, STATUS_TIMEOUT);
             *abort_flag = 1;
             return false;

@@ -48,10 +48,24 @@ class PrunedNetwork:
                 raise ValueError(how)
 
     def _prune(self):
+        # layers whose outputs meet in a residual add carry a common ``share`` tag: one ranking over the whole group,
+        # taken on the weights as given (before any slicing), and every member loses the same filters
+        shared = {}
+        for l in self.table["layers"]:
+            tag = l.get("share") if l["kind"] == "conv" else None
+            if tag is not None and l["keep"] is not None and tag not in shared:
+                members = [m for m in self.table["layers"] if m["kind"] == "conv" and m.get("share") == tag]
+                shared[tag] = B.cprune_select_shared([self.params[m["name"]][0] for m in members], l["keep"])
         for l in self.table["layers"]:
             if l["kind"] != "conv" or l["keep"] is None:
                 continue
             w, b = self.params[l["name"]]
+            if l.get("share") is not None:
+                kept = shared[l["share"]]
+                self.params[l["name"]] = (B.cprune_gather_rows(w, kept), B.cprune_gather_rows(b, kept))
+                self.kept[l["name"]] = kept
+                self._follow(l, kept, False)
+                continue
             w_next, dw = None, False
             if l["consumers"]:
                 cname, how = l["consumers"][0]
@@ -162,6 +176,20 @@ class PrunedNetwork:
         buf = self.model.copy_tensor(self.tensor_ids[name])
         torch.cuda.synchronize(self.device)
         return buf.float().cpu().numpy()[..., :c]
+
+    def task_priorities(self, reps=5):
+        """The model's tasks in the order the paper tries them for pruning (Sec. 3.3, 3.4): every distinct plan with
+        the layers (subgraphs) that share it, its measured time and its pruning impact = time x subgraphs, sorted by
+        impact.  The table comes from cprune_model_task_table, the times from cprune_model_time_tasks, the order from
+        cprune_task_order."""
+        table = self.model.task_table()
+        ms = self.model.time_tasks(reps)
+        by_handle = {}
+        for name, plan in self.plans.items():
+            by_handle.setdefault(plan.handle.value, []).append(name)
+        order = B.cprune_task_order(ms, [c for _, c, _ in table])
+        return [{"plan": self.plans[by_handle[table[j][0]][0]], "layers": by_handle[table[j][0]], "count": table[j][1],
+                 "ms": ms[j], "impact": ms[j] * table[j][1]} for j in order]
 
     def flops(self):
         return sum(p.flops for p in self.plans.values())

@@ -128,3 +128,78 @@ def test_missing_library_fails_loudly(cp, monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libcprune.so")
     with pytest.raises(RuntimeError):
         binding.lib()
+
+
+# ------------------------------------------------------------------ pruning decision, task ordering
+
+def test_prune_step_follows_the_lcm_rule_on_the_plans_own_splits(cp):
+    import oracle
+    cases = [(64, 64, 56, 56, 44, 3, 1, 1, 1), (64, 128, 28, 28, 89, 3, 1, 1, 1), (64, 256, 14, 14, 358, 3, 1, 1, 1),
+             (64, 512, 7, 7, 358, 3, 1, 1, 1), (64, 64, 56, 56, 128, 1, 2, 0, 1), (64, 320, 7, 7, 1280, 1, 1, 0, 1),
+             (64, 144, 56, 56, 144, 3, 1, 1, 144), (64, 720, 7, 7, 720, 3, 1, 1, 720), (1, 16, 8, 8, 24, 3, 1, 1, 1)]
+    for N, C, H, W, K, R, stride, pad, groups in cases:
+        p = cp.cprune_task_plan(N, C, H, W, K, R, R, stride, pad, groups)
+        want = oracle.prune_step_lcm(p.split_compute, p.split_store, p.unit_compute, p.unit_store)
+        got = cp.cprune_prune_step(p)
+        assert got == want and 1 <= got <= p.k_alloc, (N, C, K, got, want)
+        # the splits describe the plan's own tiling of the filter axis
+        prod_c = p.split_compute[0] * p.split_compute[1] * p.unit_compute
+        prod_s = p.split_store[0] * p.split_store[1] * p.unit_store
+        assert prod_c >= p.k_pad and prod_s >= p.k_pad, (N, C, K, prod_c, prod_s)
+    # one filter tile of 48 = 3 groups of 16 and 6 pieces of 8: smallest slices 16 and 8, lcm 16
+    p = cp.cprune_task_plan(64, 64, 56, 56, 44, 3, 3, 1, 1)
+    assert (p.split_compute, p.unit_compute, p.split_store, p.unit_store) == ([1, 3], 16, [1, 6], 8)
+    assert cp.cprune_prune_step(p) == 16
+
+
+def test_task_estimate_is_a_staircase_in_the_filter_count(cp):
+    p = cp.cprune_task_plan(64, 128, 28, 28, 128, 3, 3, 1, 1)
+    est = [cp.cprune_task_estimate(p, k) for k in range(128, 31, -1)]
+    assert est[0] == pytest.approx(p.est_us) and all(e > 0 for e in est)
+    assert all(a >= b - 1e-9 for a, b in zip(est, est[1:])), "fewer filters never cost more in the model"
+    levels = sorted(set(round(e, 6) for e in est))
+    assert 3 <= len(levels) <= 16, levels           # flat stretches with steps in between, not a ramp
+    with pytest.raises(cp.CpruneError) as e:
+        cp.cprune_task_estimate(p, 0)
+    assert e.value.status == 1
+    d = cp.cprune_task_plan(64, 144, 56, 56, 144, 3, 3, 1, 1, groups=144)
+    assert cp.cprune_task_estimate(d, 72) < cp.cprune_task_estimate(d, 144)
+
+
+def test_task_order_matches_the_paper_and_the_oracle(cp):
+    import oracle
+    assert cp.cprune_task_order([0.954, 0.473, 1.632], [2, 3, 1]) == [0, 2, 1]        # T1, T3, T2 (paper Sec. 3.3)
+    assert cp.cprune_task_order([], []) == []
+    import workloads as wl
+    t = list(wl.normal(77, 1, 40) ** 2)
+    c = [1 + (i * 7) % 4 for i in range(40)]
+    t[5], c[5], t[9], c[9] = 2.0, 3, 3.0, 2                                           # an exact tie: lower index first
+    assert cp.cprune_task_order(t, c) == oracle.task_order(t, c)
+
+
+def test_no_swept_shape_leaves_the_tensor_cores(cp):
+    # every dense shape of the sweep, at every kept filter count from full width to a quarter and at both batch
+    # sizes, gets a tensor-core plan; every depthwise shape a depthwise plan
+    import workloads as wl
+    for N in (1, 64):
+        for shp in wl.sweep_shapes():
+            dw = shp["groups"] > 1
+            for K in range(shp["K"], (shp["K"] + 3) // 4 - 1, -1):
+                p = cp.cprune_task_plan(N, K if dw else shp["C"], shp["H"], shp["W"], K, shp["R"], shp["S"], shp["stride"],
+                                        shp["pad"], K if dw else 1, shp["act"])
+                assert cp.KERNEL_NAMES[p.kernel] == ("depthwise" if dw else "tensor"), (N, shp, K)
+        cp.cprune_cache_clear()
+
+
+def test_plan_flags_are_part_of_the_cache_key(cp):
+    a = cp.cprune_task_plan(16, 64, 32, 32, 48, 3, 3, 1, 1)
+    b = cp.cprune_task_plan(16, 64, 32, 32, 48, 3, 3, 1, 1, flags=("im2col_only",))
+    assert a.handle.value != b.handle.value and a.variant == 1 and b.variant == 0
+    with pytest.raises(cp.CpruneError) as e:
+        L = cp.lib()
+        from paper_2207_01260_b200.binding import TaskOpts
+        import ctypes
+        h = ctypes.c_void_p()
+        st = L.cprune_task_plan(1, 8, 8, 8, 8, 3, 3, 1, 1, 1, ctypes.byref(TaskOpts(1, 0, 0, 0, 64)), ctypes.byref(h))
+        raise cp.CpruneError(st, "cprune_task_plan")
+    assert e.value.status == 1
