@@ -140,7 +140,7 @@ def main():
     ap.add_argument("--no-task-times", action="store_true",
                     help="skip the per-task timing passes (and with them the roofline object); for profiler launch lists")
     ap.add_argument("--task", default=None,
-                    help="time ONE conv task instead of a model: N,C,H,W,K,R,stride,pad[,groups[,act[,residual]]]")
+                    help="time ONE conv task instead of a model: N,C,H,W,K,R,stride,pad[,groups[,act[,residual[,pool]]]]")
     ap.add_argument("--sweep", action="store_true",
                     help="time every distinct conv shape of the four models while the kept filter count K goes "
                          "from full width down to a quarter (the staircase of latency against K)")
@@ -328,8 +328,9 @@ def task_bench(args):
     groups = int(f[8]) if len(f) > 8 else 1
     act = f[9] if len(f) > 9 else "relu"
     residual = len(f) > 10 and f[10] == "1"
+    pool = f[11] if len(f) > 11 and f[11] not in ("", "none") else None
     torch.cuda.set_device(0)
-    plan = cp.cprune_task_plan(N, C, H, W, K, R, R, stride, pad, groups, act, residual)
+    plan = cp.cprune_task_plan(N, C, H, W, K, R, R, stride, pad, groups, act, residual, pool)
     i = plan.info
     x, w, b, res = wl.conv_task_tensors(7, N, C, H, W, K, R, R, groups, residual, i["P"], i["Q"])
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()

@@ -172,7 +172,7 @@ typedef struct {
 
 /* Host only; launches nothing.  opts == NULL means bias + ReLU, no residual, no pool, AUTO.
  * Plans are cached: an identical (shape, opts) key returns the same handle with its reference
- * count raised.  groups must be 1 or C (depthwise; then K == C and R == S == 3).
+ * count raised.  groups must be 1 or C (depthwise; then K == C and R == S == 3 or 5, stride 1 or 2).
  * The pool option (paper Sec. 3.4: a task is the fused subgraph) is applied to the activated result:
  * CPRUNE_POOL_MAX2X2 needs even P and Q; CPRUNE_POOL_MAX3X3S2 (3x3, stride 2, pad 1) takes any extent.
  * Errors: INVALID_ARG (non-positive extents, output extent < 1, 2x2 pool on odd P/Q), UNSUPPORTED. */

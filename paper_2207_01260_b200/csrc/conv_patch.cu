@@ -495,6 +495,13 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const bool clamp_lo = p.act != CPRUNE_ACT_NONE;      // results are >= 0
         const bool store_thread = warp == PK_FIRST_EPI && lane == 0;
         const int groups = (p.FT + 63) / 64;
+        // one group and one filter tile: a thread stages the same 32 filters in every tile and keeps their bias in registers
+        const bool bias_const = !DENSE && groups == 1 && p.tiles_n == 1;
+        float bias_r[32];
+        if (bias_const) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) bias_r[j] = (half * 32 + j < p.FT) ? __ldg(p.bias + half * 32 + j) : 0.f;
+        }
         const int n_entries = p.pool == 1 ? (p.TH >> 1) * (p.Q >> 1) : ((p.TH - 1) >> 1) * ((p.TW - 1) >> 1);
         // 3x3 pool: a thread copies out at most two (pooled pixel, 8 filters) items per tile, the same ones in every tile;
         // the shared-memory offsets of their nine window slots are worked out once
@@ -514,20 +521,10 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 }
             }
         }
-        // The residual of a group arrives by TMA in the staging buffer the group will use (same box as the store:
-        // wrap-around slots read as zero); the values are added there in place.  The load for the next group is
-        // issued as soon as its buffer is free.
-        const bool with_res = p.res != nullptr;
-        auto load_residual = [&](int item_, int g_, uint32_t counter) {
-            int tm_ = item_, nt_ = 0;
-            if (p.tiles_n > 1) { tm_ = item_ / p.tiles_n; nt_ = item_ - tm_ * p.tiles_n; }
-            int n_, p0_, q0_;
-            tile_origin(p, tm_, n_, p0_, q0_);
-            const uint32_t b = p.staging_bufs == 2 ? (counter & 1u) : 0u;
-            mbar_expect_tx(res_full(b), (uint32_t)(p.TH * p.Wp * 128));
-            tma_load_4d(staging0 + b * stage_buf_bytes, &tm_res, res_full(b), nt_ * p.FT + g_ * 64, q0_, p0_, n_);
-        };
-        // dense staging: the residual of tile item_ (tiles_n == 1, one row of tiles) is one contiguous range as well
+        // Residuals.  Everywhere but with dense staging the MMA warps add the residual on the tensor core (see there) and
+        // the epilogue has nothing to do with it.  Dense staging: the residual of tile item_ (tiles_n == 1, one row of
+        // tiles) is one contiguous range of memory, arrives in the staging buffer the tile will use and is added in place.
+        const bool with_res = DENSE && p.res != nullptr;
         auto load_residual_dense = [&](int item_, uint32_t counter) {
             const int q0_ = item_ * p.step_w;
             const uint32_t bytes = (uint32_t)min(p.TW, p.Q - q0_) * (uint32_t)p.k_pad * 2u;
@@ -537,8 +534,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         };
         if (with_res && store_thread && (int)blockIdx.x < total_items) {
             pdl_wait();        // the residual is the result of an earlier kernel of the chain
-            if constexpr (DENSE) load_residual_dense(blockIdx.x, 0);
-            else load_residual(blockIdx.x, 0, 0);
+            load_residual_dense(blockIdx.x, 0);
         }
         for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
             int tm = item, nt = 0;
@@ -627,53 +623,57 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     ok = __all_sync(0xffffffffu, mbar_wait(sempty(group_counter & 1u), ((group_counter >> 1) & 1u) ^ 1u, abort_flag, p.status, false));
                     if (!ok) break;
                 }
-                if (with_res) {
-                    const uint32_t b = p.staging_bufs == 2 ? (group_counter & 1u) : 0u;
-                    const uint32_t par = p.staging_bufs == 2 ? ((group_counter >> 1) & 1u) : (group_counter & 1u);
-                    ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), par, abort_flag, p.status, false));
-                    if (!ok) break;
-                }
-                for (int mb = 0; mb < p.MT; ++mb) {
-                    uint32_t v[32];
+                // Units of 16 filters of one accumulator block: (block 0, first 16), (block 0, second 16), (block 1, ...).
+                // The tensor-memory load of unit u + 1 is in flight while unit u is turned into bf16 and staged, so that
+                // only the first load's latency is exposed; two register buffers alternate.
+                const bool u_ok[4] = {ch < p.FT, ch + 16 < p.FT, p.MT == 2 && ch < p.FT, p.MT == 2 && ch + 16 < p.FT};
+                auto unit_addr = [&](int u) { return t_row + (uint32_t)((u >> 1) * p.FT + ch + (u & 1) * 16); };
+                auto stage_unit = [&](int u, const uint32_t *v) {
+                    const int c0 = ch + (u & 1) * 16;
+                    float f[16];
+                    if (bias_const) {
 #pragma unroll
-                    for (int sb = 0; sb < 2; ++sb)
-                        if (ch + sb * 16 < p.FT) tmem_ld16(t_row + (uint32_t)(mb * p.FT + ch + sb * 16), v + sb * 16);
-                    bf16x8 rv[4];
-                    if (with_res) {
+                        for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(v[j]) + bias_r[(u & 1) * 16 + j];
+                    } else {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            rv[j] = *(const bf16x8 *)(buf + mb * PK_BLOCK_BYTES + sub_off(trow, half * 4 + j));
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 b4 = *(const float4 *)(bias_src + k0 + c0 + q * 4);
+                            f[q * 4 + 0] = __uint_as_float(v[q * 4 + 0]) + b4.x;
+                            f[q * 4 + 1] = __uint_as_float(v[q * 4 + 1]) + b4.y;
+                            f[q * 4 + 2] = __uint_as_float(v[q * 4 + 2]) + b4.z;
+                            f[q * 4 + 3] = __uint_as_float(v[q * 4 + 3]) + b4.w;
+                        }
                     }
+                    if (p.act == CPRUNE_ACT_RELU) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) f[j] = fmaxf(f[j], 0.f);
+                    } else if (p.act == CPRUNE_ACT_RELU6) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) f[j] = fminf(fmaxf(f[j], 0.f), 6.f);
+                    }
+                    uint8_t *blk = buf + (u >> 1) * PK_BLOCK_BYTES;
+                    *(bf16x8 *)(blk + sub_off(trow, half * 4 + (u & 1) * 2)) = pack8(f);
+                    *(bf16x8 *)(blk + sub_off(trow, half * 4 + (u & 1) * 2 + 1)) = pack8(f + 8);
+                };
+                {
+                    uint32_t va[16], vb[16];
+                    if (u_ok[0]) tmem_ld16(unit_addr(0), va);
                     tmem_ld_wait();
-                    if (g == groups - 1 && mb == p.MT - 1) {     // accumulator fully read: hand it back
+                    if (u_ok[1]) tmem_ld16(unit_addr(1), vb);
+                    if (u_ok[0]) stage_unit(0, va);
+                    tmem_ld_wait();
+                    if (u_ok[2]) tmem_ld16(unit_addr(2), va);
+                    if (u_ok[1]) stage_unit(1, vb);
+                    tmem_ld_wait();
+                    if (u_ok[3]) tmem_ld16(unit_addr(3), vb);
+                    if (u_ok[2]) stage_unit(2, va);
+                    tmem_ld_wait();
+                    if (g == groups - 1) {     // accumulator fully read: hand it back
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(tempty(acc));
                     }
-#pragma unroll
-                    for (int sb = 0; sb < 2; ++sb) {
-                        const int c0 = ch + sb * 16;
-                        if (c0 < p.FT) {
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                float f[8];
-                                const float4 b0 = *(const float4 *)(bias_src + k0 + c0 + h * 8);
-                                const float4 b1 = *(const float4 *)(bias_src + k0 + c0 + h * 8 + 4);
-                                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[sb * 16 + h * 8 + j]) + bb[j];
-                                if (with_res) {
-                                    float rf[8];
-                                    unpack8(rv[sb * 2 + h], rf);
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j) f[j] += rf[j];
-                                }
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) f[j] = fminf(fmaxf(f[j], act_lo), act_hi);
-                                *(bf16x8 *)(buf + mb * PK_BLOCK_BYTES + sub_off(trow, half * 4 + sb * 2 + h)) = pack8(f);
-                            }
-                        }
-                    }
+                    if (u_ok[3]) stage_unit(3, vb);
                 }
                 if constexpr (SPLIT) {
                     // hand the staged group to the pooling warps and go on with the next one
@@ -695,13 +695,6 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                         if (k0 + g * 64 < p.k_pad) tma_store_4d(&tm_y, staging0 + boff, k0 + g * 64, q0, p0, n);
                         tma_store_commit();
                         if (p.staging_bufs == 1) tma_store_wait_read<0>();
-                        if (with_res) {
-                            // next group of this CTA: its buffer is free (two buffers: its last store was waited for
-                            // before the barrier above; one buffer: just now)
-                            int ni = item, ng = g + 1;
-                            if (ng == groups) { ni = item + gridDim.x; ng = 0; }
-                            if (ni < total_items) load_residual(ni, ng, group_counter + 1);
-                        }
                     }
                     if (p.staging_bufs == 1) {
                         ok = epi_sync();
@@ -928,7 +921,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             // tiles long, so the ring is as deep as fits)
             int ps_max = 2;
             if (cblks > 2 && patch_bytes <= 32 * 1024) ps_max = cblks < PK_MAX_PATCH_STAGES ? cblks : PK_MAX_PATCH_STAGES;
-            if (g.flat) ps_max = PK_MAX_PATCH_STAGES;
+            if (g.flat || g.stem) ps_max = PK_MAX_PATCH_STAGES;     // (stems: a tile is a few MMAs, shorter than a load's latency)
             // A residual travels through the patch ring too (64 filters per stage).  A deeper ring, which would let the
             // next tile's first patch be fetched while the residual blocks are still in use, was measured against the
             // shallow one with the shared memory spent on resident filters / more filter stages instead: the shallow ring

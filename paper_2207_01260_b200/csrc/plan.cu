@@ -166,7 +166,7 @@ cprune_status cprune_task_plan(int N, int C, int H, int W, int K, int R, int S, 
         return CPRUNE_ERR_INVALID_ARG;
     if (groups != 1) {
         if (groups != C || K != C) return CPRUNE_ERR_UNSUPPORTED;
-        if (R != 3 || S != 3 || stride > 2) return CPRUNE_ERR_UNSUPPORTED;
+        if (R != S || (R != 3 && R != 5) || stride > 2) return CPRUNE_ERR_UNSUPPORTED;
     }
     int P = (H + 2 * pad - R) / stride + 1, Q = (W + 2 * pad - S) / stride + 1;
     if (o.pool == CPRUNE_POOL_MAX2X2 && ((P & 1) || (Q & 1))) return CPRUNE_ERR_INVALID_ARG;

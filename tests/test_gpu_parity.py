@@ -439,6 +439,15 @@ def test_depthwise_task_parity(cp, C, H, W, stride):
     assert cp.KERNEL_NAMES[plan.kernel] == "depthwise"
 
 
+@pytest.mark.parametrize("C,H,W,stride", [(72, 56, 56, 2), (120, 28, 28, 1), (90, 17, 15, 2), (576, 14, 14, 2), (1152, 7, 7, 1),
+                                          (8, 6, 5, 1), (20, 3, 2, 1)])
+def test_depthwise_5x5_task_parity(cp, C, H, W, stride):
+    # MnasNet's 5x5 depthwise layers (pad 2): ragged tiles, channel counts off the 8 / 64 grid, images smaller than the filter
+    plan = check_task(cp, 2, C, H, W, C, 5, stride, 2, groups=C, act="relu")
+    assert cp.KERNEL_NAMES[plan.kernel] == "depthwise"
+    check_task(cp, 1, C, H, W, C, 5, stride, 2, groups=C, act="none", with_res=(stride == 1))
+
+
 def test_task_runs_are_deterministic(cp):
     x, w, b, _ = wl.conv_task_tensors(5, 2, 89, 14, 14, 128, 3, 3)
     plan = cp.cprune_task_plan(2, 89, 14, 14, 128, 3, 3, 1, 1)
@@ -588,6 +597,14 @@ def test_model_parity_at_the_benchmarked_batch(cp, name, batch, oracle_images):
     net, _, _ = model_parity(cp, name, batch, oracle_images=oracle_images)
     kinds = {cp.KERNEL_NAMES[i["kernel"]] for i in net.conv_launch_info().values()}
     assert "direct" not in kinds
+
+
+def test_mnasnet_parity(cp):
+    net, _, _ = model_parity(cp, "mnasnet1_0", 2)
+    kinds = {cp.KERNEL_NAMES[i["kernel"]] for i in net.conv_launch_info().values()}
+    assert kinds == {"tensor", "depthwise"}
+    assert {net.plans[n].R for n in net.plans if n.endswith("_dw")} == {3, 5}
+    model_parity(cp, "mnasnet1_0", 16, hw=96, oracle_images=4)
 
 
 def test_shared_selection_and_shortcut_pruned_resnet(cp):

@@ -115,7 +115,7 @@ def test_plan_argument_errors(cp):
             cp.cprune_task_plan(*args)
         assert e.value.status == 1
     with pytest.raises(cp.CpruneError) as e:
-        cp.cprune_task_plan(1, 8, 8, 8, 8, 5, 5, 1, 2, groups=8)      # depthwise is 3x3 only
+        cp.cprune_task_plan(1, 8, 8, 8, 8, 7, 7, 1, 3, groups=8)      # depthwise is 3x3 or 5x5
     assert e.value.status == 2
     with pytest.raises(cp.CpruneError) as e:
         cp.cprune_task_plan(1, 8, 7, 7, 8, 3, 3, 1, 1, pool="max2x2")  # odd extent cannot be pooled 2x2

@@ -345,10 +345,10 @@ def conv_task_tensors(seed: int, N, C, H, W, K, R, S, groups=1, with_res=False, 
 
 
 def sweep_shapes() -> list:
-    """The distinct full-width conv task shapes of the four models, as dicts
+    """The distinct full-width conv task shapes of the models (MnasNet1.0 adds its 5x5 depthwise layers), as dicts
     {C, K, H, W, R, S, stride, pad, groups, act}; depthwise shapes have groups == C == K."""
     seen, out = set(), []
-    for fn in (single_task, vgg16_cifar, resnet18, mobilenet_v2):
+    for fn in (single_task, vgg16_cifar, resnet18, mobilenet_v2, mnasnet1_0):
         m = fn()
         sz = spatial_sizes(m)
         for l in m["layers"]:
