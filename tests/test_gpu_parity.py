@@ -258,17 +258,8 @@ def test_stride_1_tasks_on_the_im2col_kernel(cp):
 
 
 def big_task_tensors(seed, N, C, H, W, K, R, groups, with_res, P, Q, base=4):
-    """Tensors of a full-size task.  Drawing every image from the generator would take minutes over a whole model, so
-    `base` images are drawn and image n is image n % base scaled by 1 + n / 256 (exact in float32 for these n): all
-    images differ, so an output written to the wrong image shows."""
-    nb = min(N, base)
-    x, w, b, res = wl.conv_task_tensors(seed, nb, C, H, W, K, R, R, groups, with_res, P, Q)
-    scale = (1.0 + np.arange(N, dtype=np.float32) / 256.0).reshape(N, 1, 1, 1)
-    idx = np.arange(N) % nb
-    x = np.ascontiguousarray(x[idx] * scale)
-    if res is not None:
-        res = np.ascontiguousarray(res[idx] * scale)
-    return x, w, b, res
+    """Tensors of a full-size task (drawing every image from the generator would take minutes over a whole model)."""
+    return wl.conv_task_tensors_tiled(seed, N, C, H, W, K, R, R, groups, with_res, P, Q, base)
 
 
 def sample_points(rng, N, oh, ow, K, n_pts):

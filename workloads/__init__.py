@@ -344,6 +344,20 @@ def conv_task_tensors(seed: int, N, C, H, W, K, R, S, groups=1, with_res=False, 
     return x, w, b, res
 
 
+def conv_task_tensors_tiled(seed: int, N, C, H, W, K, R, S, groups=1, with_res=False, P=None, Q=None, base=4):
+    """The tensors of conv_task_tensors for a LARGE batch without drawing every image: `base` images are drawn
+    and image n is image n % base scaled by 1 + n / 256 (exact in float32 for n < 2^15), so that all images differ
+    and an output written to the wrong image shows.  Input generation only: no part of the method."""
+    nb = min(N, base)
+    x, w, b, res = conv_task_tensors(seed, nb, C, H, W, K, R, S, groups, with_res, P, Q)
+    scale = (1.0 + np.arange(N, dtype=np.float32) / 256.0).reshape(N, 1, 1, 1)
+    idx = np.arange(N) % nb
+    x = np.ascontiguousarray(x[idx] * scale)
+    if res is not None:
+        res = np.ascontiguousarray(res[idx] * scale)
+    return x, w, b, res
+
+
 def sweep_shapes() -> list:
     """The distinct full-width conv task shapes of the models (MnasNet1.0 adds its 5x5 depthwise layers), as dicts
     {C, K, H, W, R, S, stride, pad, groups, act}; depthwise shapes have groups == C == K."""
