@@ -239,10 +239,45 @@ cprune_status cprune_fc(const void *x, int N, int in, const void *w_packed, cons
                         int out_is_f32, void *y, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Fused inverted-residual block (the MobileNetV2 / MnasNet building block of the paper's Sec. 4.1 models): the three
+ * tasks 1x1 expand + activation, 3x3 depthwise (stride 1, pad 1) + activation, 1x1 project (+ the block's input as
+ * residual, then act_out) run as ONE kernel that keeps the expanded tensor on the SM.  The result equals that of the
+ * three tasks run one after the other (bf16 is rounded at the same places).
+ *   x  device bf16 [N][H][W][c_in_pad]        y  device bf16 [N][H][W][k_pad]
+ * Supported: stride 1, H * W <= 256 and (H + 2) * (W + 2) <= 256 (one image per thread block), C_in <= 192,
+ * C_out <= 256 (<= 192 when H * W > 128); anything else returns CPRUNE_ERR_UNSUPPORTED and the caller runs the three
+ * tasks separately.  residual != 0 requires C_in == C_out.  Plans are cached and reference-counted like task plans.
+ * cprune_block_pack: float32 w_expand [hidden][C_in], w_depthwise [hidden][1][3][3], w_project [C_out][hidden] and the
+ * three biases (each may be NULL = zeros) -> one packed bf16 buffer and one packed float32 bias buffer. */
+typedef struct cprune_block cprune_block;
+typedef struct {
+    int N, C_in, H, W, hidden, C_out, act, act_out, residual;
+    int c_in_pad, k_pad, hid_alloc, k_alloc;
+    size_t packed_weight_bytes, packed_bias_bytes;
+    double flops;               /* 2 N H W (C_in hidden + 9 hidden + hidden C_out) */
+    double algorithmic_bytes;   /* x + y + parameters, each once */
+    double unfused_bytes;       /* the same with the expanded tensor written and read by three separate tasks */
+    int splits;                 /* thread blocks per image (each takes a share of the hidden channels); > 1 adds a second launch */
+    size_t workspace_bytes;     /* float32 partial sums of the project layer when splits > 1 */
+    double est_us;              /* the planner's estimate (microseconds) */
+} cprune_block_info;
+cprune_status cprune_block_plan(int N, int C_in, int H, int W, int hidden, int C_out, int act, int act_out, int residual,
+                                cprune_block **out);
+cprune_status cprune_block_query(const cprune_block *block, cprune_block_info *out /* host */);
+cprune_status cprune_block_release(cprune_block *block);
+cprune_status cprune_block_pack(const cprune_block *block, const float *w_expand, const float *b_expand, const float *w_depthwise,
+                                const float *b_depthwise, const float *w_project, const float *b_project, void *w_packed,
+                                float *b_packed, void *stream);
+/* Enqueue only (at most two launches), no allocation.  Pointers 16-byte aligned; workspace (device, workspace_bytes) may be
+ * NULL when the plan needs none. */
+cprune_status cprune_block_run(cprune_block *block, const void *x, const void *w_packed, const float *b_packed, void *y, void *workspace,
+                               void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Whole models: the aggregate of a network's tasks run back to back (paper Sec. 3.1: the model
  * is compiled as the aggregate of its tasks' programs, and its execution time is measured).
  */
-enum { CPRUNE_OP_CONV = 1, CPRUNE_OP_MAXPOOL = 2, CPRUNE_OP_GAP = 3, CPRUNE_OP_FC = 4 };
+enum { CPRUNE_OP_CONV = 1, CPRUNE_OP_MAXPOOL = 2, CPRUNE_OP_GAP = 3, CPRUNE_OP_FC = 4, CPRUNE_OP_BLOCK = 5 };
 
 typedef struct {
     int op;                 /* CPRUNE_OP_* */
@@ -251,6 +286,8 @@ typedef struct {
     const void *w;          /* CONV / FC: packed weights, device, borrowed */
     const float *b;         /* CONV / FC: packed bias, device, borrowed */
     int p0, p1, p2, p3;     /* MAXPOOL: k, stride, pad, -.  FC: in_features, out_features, activation, - */
+    cprune_block *block;    /* BLOCK: the fused block's plan (borrowed); w and b are its packed buffers, res is unused
+                               (the block's residual is its own input) */
 } cprune_task_desc;
 
 /* Builds a model for input float32 [N][H][W][C].  tasks is a host array, copied.  The output of the

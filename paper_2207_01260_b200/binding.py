@@ -19,7 +19,7 @@ POOL = {None: 0, "none": 0, "max2x2": 1, "max3x3s2": 2}
 KERNEL = {"auto": 0, "direct": 1, "tensor": 2, "depthwise": 3}
 KERNEL_NAMES = {v: k for k, v in KERNEL.items()}
 FLAGS = {"im2col_only": 1, "pool_on_epilogue_warps": 2}
-OP_CONV, OP_MAXPOOL, OP_GAP, OP_FC = 1, 2, 3, 4
+OP_CONV, OP_MAXPOOL, OP_GAP, OP_FC, OP_BLOCK = 1, 2, 3, 4, 5
 
 # every symbol include/cprune.h declares
 EXPORTS = [
@@ -30,7 +30,8 @@ EXPORTS = [
     "cprune_fc", "cprune_model_create", "cprune_model_run", "cprune_model_run_host", "cprune_model_tensor", "cprune_model_copy_tensor", "cprune_model_launches",
     "cprune_model_destroy", "cprune_poll_device_status", "cprune_select_shared", "cprune_prune_step",
     "cprune_task_estimate", "cprune_task_order", "cprune_model_task_table", "cprune_model_time_tasks",
-    "cprune_selftest_wait_timeout",
+    "cprune_selftest_wait_timeout", "cprune_block_plan", "cprune_block_query", "cprune_block_release", "cprune_block_pack",
+    "cprune_block_run",
 ]
 
 
@@ -65,7 +66,15 @@ class TaskEntry(ctypes.Structure):
 
 class TaskDesc(ctypes.Structure):
     _fields_ = [("op", c_int), ("in_", c_int), ("out", c_int), ("res", c_int), ("plan", c_void_p), ("w", c_void_p),
-                ("b", c_void_p), ("p0", c_int), ("p1", c_int), ("p2", c_int), ("p3", c_int)]
+                ("b", c_void_p), ("p0", c_int), ("p1", c_int), ("p2", c_int), ("p3", c_int), ("block", c_void_p)]
+
+
+class BlockInfo(ctypes.Structure):
+    _fields_ = [(n, c_int) for n in ("N", "C_in", "H", "W", "hidden", "C_out", "act", "act_out", "residual", "c_in_pad", "k_pad",
+                                      "hid_alloc", "k_alloc")] + \
+               [("packed_weight_bytes", c_size_t), ("packed_bias_bytes", c_size_t), ("flops", c_double),
+                ("algorithmic_bytes", c_double), ("unfused_bytes", c_double), ("splits", c_int), ("workspace_bytes", c_size_t),
+                ("est_us", c_double)]
 
 
 _lib = None
@@ -119,6 +128,11 @@ def lib():
         L.cprune_model_task_table.argtypes = [c_void_p, POINTER(TaskEntry), c_int, POINTER(c_int)]
         L.cprune_model_time_tasks.argtypes = [c_void_p, c_int, POINTER(c_double), c_void_p]
         L.cprune_selftest_wait_timeout.argtypes = [c_void_p]
+        L.cprune_block_plan.argtypes = [c_int] * 9 + [POINTER(c_void_p)]
+        L.cprune_block_query.argtypes = [c_void_p, POINTER(BlockInfo)]
+        L.cprune_block_release.argtypes = [c_void_p]
+        L.cprune_block_pack.argtypes = [c_void_p] * 10
+        L.cprune_block_run.argtypes = [c_void_p] * 7
         _lib = L
     return _lib
 
@@ -329,6 +343,57 @@ def cprune_task_run(plan: Plan, x, w_packed, b_packed, residual=None, y=None, wo
     return y
 
 
+class Block:
+    """Handle of a cached fused-block plan (released when collected)."""
+
+    def __init__(self, handle):
+        self.handle = handle
+        info = BlockInfo()
+        _check(lib().cprune_block_query(handle, byref(info)), "cprune_block_query")
+        self.info = {n: getattr(info, n) for n, _ in info._fields_}
+
+    def __del__(self):
+        try:
+            if self.handle and _lib is not None:
+                _lib.cprune_block_release(self.handle)
+        except Exception:
+            pass
+
+    def __getattr__(self, name):
+        info = self.__dict__.get("info", {})
+        if name in info:
+            return info[name]
+        raise AttributeError(name)
+
+
+def cprune_block_plan(N, C_in, H, W, hidden, C_out, activation="relu6", act_out="none", residual=False) -> Block:
+    h = c_void_p()
+    _check(lib().cprune_block_plan(N, C_in, H, W, hidden, C_out, ACT[activation], ACT[act_out], 1 if residual else 0, byref(h)),
+           "cprune_block_plan")
+    return Block(h)
+
+
+def cprune_block_pack(block: Block, w_expand, b_expand, w_depthwise, b_depthwise, w_project, b_project, stream=None):
+    dev = w_expand.device
+    wp = torch.empty(block.packed_weight_bytes // 2, dtype=torch.bfloat16, device=dev)
+    bp = torch.empty(block.packed_bias_bytes // 4, dtype=torch.float32, device=dev)
+    _check(lib().cprune_block_pack(block.handle, _ptr(_dev_f32(w_expand)), _ptr(b_expand), _ptr(_dev_f32(w_depthwise)),
+                                   _ptr(b_depthwise), _ptr(_dev_f32(w_project)), _ptr(b_project), _ptr(wp), _ptr(bp),
+                                   _stream(stream)), "cprune_block_pack")
+    return wp, bp
+
+
+def cprune_block_run(block: Block, x, w_packed, b_packed, y=None, workspace=None, stream=None):
+    """x bf16 [N,H,W,c_in_pad] -> y bf16 [N,H,W,k_pad]."""
+    if y is None:
+        y = torch.empty((block.N, block.H, block.W, block.k_pad), dtype=torch.bfloat16, device=x.device)
+    if workspace is None and block.workspace_bytes:
+        workspace = torch.empty(block.workspace_bytes, dtype=torch.uint8, device=x.device)
+    _check(lib().cprune_block_run(block.handle, _ptr(x), _ptr(w_packed), _ptr(b_packed), _ptr(y), _ptr(workspace), _stream(stream)),
+           "cprune_block_run")
+    return y
+
+
 def cprune_cast_input(x, y=None, stream=None):
     """float32 [N,H,W,C] -> bf16 [N,H,W,c_pad]."""
     x = _dev_f32(x)
@@ -467,4 +532,4 @@ def cprune_selftest_wait_timeout(stream=None):
 
 __all__ = [n for n in dir() if n.startswith("cprune_")] + ["Plan", "Model", "TaskDesc", "CpruneError", "lib",
                                                            "EXPORTS", "KERNEL_NAMES", "OP_CONV", "OP_MAXPOOL",
-                                                           "OP_GAP", "OP_FC"]
+                                                           "OP_GAP", "OP_FC", "OP_BLOCK", "Block"]

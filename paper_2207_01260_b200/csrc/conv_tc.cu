@@ -984,6 +984,14 @@ static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w
     return CPRUNE_OK;
 }
 
+cprune_status launch_splitk_finalize(const float *partial, int splits, long long M, int k_alloc, int k_pad, const float *bias,
+                                     const void *res, int act, void *y, cudaStream_t st) {
+    const long long threads = M * (k_pad / 8) * 4;
+    CPRUNE_CUDA_CHECK(launch_chained(splitk_finalize_kernel, dim3((unsigned)ceil_div(threads, 256)), dim3(256), 0, st, partial, splits, M,
+                                     k_alloc, k_pad / 8, bias, (const bf16x8 *)res, act, 0, (bf16x8 *)y));
+    return CPRUNE_OK;
+}
+
 static int sm_count() {
     static int n = 0;
     if (!n) {

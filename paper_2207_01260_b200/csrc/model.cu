@@ -86,6 +86,9 @@ static cprune_status enqueue_chain(cprune_model *m, const float *x, float *logit
                 s = task_run_internal(d.plan, pin, d.w, d.b, d.res >= 0 ? tensor_ptr(m, d.res) : nullptr, pout, m->workspace, st,
                                       t == 0 && direct);
                 break;
+            case CPRUNE_OP_BLOCK:
+                s = cprune_block_run(d.block, pin, d.w, d.b, pout, m->workspace, st);
+                break;
             case CPRUNE_OP_MAXPOOL:
                 s = cprune_maxpool(pin, in.n, in.h, in.w, in.c, d.p0, d.p1, d.p2, pout, st);
                 break;
@@ -147,6 +150,18 @@ cprune_status cprune_model_create(int N, int H, int W, int C, const cprune_task_
                 if (i.workspace_bytes > m->workspace_bytes) m->workspace_bytes = i.workspace_bytes;
                 m->launches += ((d.plan->opts.pool && !(i.kernel == CPRUNE_KERNEL_TENSOR && d.plan->fused_pool)) ? 2 : 1) + (d.plan->splits > 1 ? 1 : 0) +
                                ((d.plan->patch && d.plan->narrow) ? 1 : 0);
+                break;
+            }
+            case CPRUNE_OP_BLOCK: {
+                if (!d.block || !d.w || !d.b) { st = CPRUNE_ERR_INVALID_ARG; break; }
+                cprune_block_info bi;
+                if (cprune_block_query(d.block, &bi) != CPRUNE_OK || bi.N != in.n || bi.H != in.h || bi.W != in.w || bi.C_in != in.c) {
+                    st = CPRUNE_ERR_INVALID_ARG;
+                    break;
+                }
+                o.h = bi.H; o.w = bi.W; o.c = bi.C_out;
+                if (bi.workspace_bytes > m->workspace_bytes) m->workspace_bytes = bi.workspace_bytes;
+                m->launches += bi.splits > 1 ? 2 : 1;
                 break;
             }
             case CPRUNE_OP_MAXPOOL:

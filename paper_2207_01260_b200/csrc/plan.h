@@ -88,6 +88,10 @@ cprune_status encode_tiled_bf16_swz(CUtensorMap *map, const void *ptr, int rank,
 // tiled bf16 tensor map without swizzle, out-of-bounds elements read as zero
 cprune_status encode_tiled_bf16(CUtensorMap *map, const void *ptr, int rank, const unsigned long long *dims,
                                 const unsigned long long *strides_bytes, const unsigned *box);
+// adds the float32 partial sums [splits][M][k_alloc] of a split reduction in index order, then bias, residual (bf16 [M][k_pad]
+// or NULL) and activation; y bf16 [M][k_pad]
+cprune_status launch_splitk_finalize(const float *partial, int splits, long long M, int k_alloc, int k_pad, const float *bias,
+                                     const void *res, int act, void *y, cudaStream_t st);
 // 2x2 stride-2 max-pool as a separate pass (used when a plan asks for a pool and the conv kernel
 // does not fuse it): x [N][H][W][c] -> y [N][H/2][W/2][c]
 cprune_status launch_maxpool(const void *x, int N, int H, int W, int c_pad, int k, int stride, int pad, void *y,

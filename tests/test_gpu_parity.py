@@ -598,6 +598,96 @@ def test_mnasnet_parity(cp):
     model_parity(cp, "mnasnet1_0", 16, hw=96, oracle_images=4)
 
 
+def block_tensors(seed, N, C_in, H, W, hidden, C_out):
+    x = wl.normal_f32(seed, 0, (N, H, W, C_in))
+    we = wl.normal_f32(seed, 1, (hidden, C_in, 1, 1), np.sqrt(2.0 / C_in))
+    wd = wl.normal_f32(seed, 2, (hidden, 1, 3, 3), np.sqrt(2.0 / 9))
+    wp = wl.normal_f32(seed, 3, (C_out, hidden, 1, 1), np.sqrt(2.0 / hidden))
+    be, bd, bp = (wl.normal_f32(seed, 4 + j, (n,), 0.05) for j, n in enumerate((hidden, hidden, C_out)))
+    return x, we, be, wd, bd, wp, bp
+
+
+def block_reference(t, act, act_out, residual, matched):
+    """The block as the chain of its three tasks in the oracle; matched: bf16 where the device rounds to bf16."""
+    x, we, be, wd, bd, wp, bp = t
+    rnd = oracle.round_bf16 if matched else (lambda a: np.asarray(a, dtype=np.float64))
+    xr = rnd(x)
+    h1 = rnd(oracle.conv2d(xr, rnd(we), be, 1, 0, 1, act))
+    h2 = rnd(oracle.conv2d(h1, rnd(wd), bd, 1, 1, wd.shape[0], act))
+    return oracle.conv2d(h2, rnd(wp), bp, 1, 0, 1, act_out, xr if residual else None, with_bound=True)
+
+
+@pytest.mark.parametrize("case", [
+    # N, C_in, H, W, hidden, C_out, act, residual: the stride-1 blocks of pruned MobileNetV2 at 14x14 and 7x7, then ragged
+    # extents, channel counts off the 8 / 16 / 64 grid, one and several 64-channel chunks, relu (MnasNet) and no activation
+    (3, 64, 14, 14, 288, 64, "relu6", True), (2, 64, 14, 14, 288, 96, "relu6", False), (2, 96, 14, 14, 432, 96, "relu6", True),
+    (4, 160, 7, 7, 720, 160, "relu6", True), (2, 24, 9, 11, 100, 40, "relu", False), (1, 75, 13, 14, 75, 75, "none", True),
+    (5, 8, 5, 4, 30, 12, "relu6", False), (2, 130, 12, 12, 64, 130, "relu", True), (1, 40, 7, 7, 200, 250, "relu", False)])
+def test_fused_inverted_residual_block(cp, case):
+    N, C_in, H, W, hidden, C_out, act, residual = case
+    t = block_tensors(61, N, C_in, H, W, hidden, C_out)
+    x, we, be, wd, bd, wp, bp = t
+    blk = cp.cprune_block_plan(N, C_in, H, W, hidden, C_out, act, "none", residual)
+    wq, bq = cp.cprune_block_pack(blk, _dev(we.reshape(hidden, C_in)), _dev(be), _dev(wd.reshape(hidden, 9)), _dev(bd),
+                                  _dev(wp.reshape(C_out, hidden)), _dev(bp))
+    y = cp.cprune_block_run(blk, cp.cprune_cast_input(_dev(x)), wq, bq).float().cpu().numpy()
+    cp.cprune_poll_device_status()
+    assert y.shape == (N, H, W, blk.k_pad) and np.all(y[..., C_out:] == 0)
+    ref, bound = block_reference(t, act, "none", residual, matched=False)
+    ref_m, bound_m = block_reference(t, act, "none", residual, matched=True)
+    got = y[..., :C_out]
+    r1 = float(np.max(np.abs(got - ref) / bound))
+    # against the matched chain: the stored result's own rounding, plus what a differently rounded hidden value (float32
+    # against float64 sums under the two bf16 roundings inside the block) can move: far below 1e-3 of the scale
+    r2 = float(np.max(np.abs(got - ref_m) / (MATCH_REL * np.abs(ref_m) + 1e-3 * bound_m)))
+    WORST["fused block %s" % (case,)] = (r1, r2)
+    assert r1 <= TOL and r2 <= 1.0, (case, r1, r2)
+    # the same three tasks run separately give the same values up to those rounding flips
+    p1 = cp.cprune_task_plan(N, C_in, H, W, hidden, 1, 1, 1, 0, 1, act)
+    p2 = cp.cprune_task_plan(N, hidden, H, W, hidden, 3, 3, 1, 1, hidden, act)
+    p3 = cp.cprune_task_plan(N, hidden, H, W, C_out, 1, 1, 1, 0, 1, "none", residual)
+    xb = cp.cprune_cast_input(_dev(x))
+    a = cp.cprune_task_run(p1, xb, *cp.cprune_pack_weights(p1, _dev(we), _dev(be)))
+    b = cp.cprune_task_run(p2, a, *cp.cprune_pack_weights(p2, _dev(wd), _dev(bd)))
+    c = cp.cprune_task_run(p3, b, *cp.cprune_pack_weights(p3, _dev(wp), _dev(bp)), xb if residual else None)
+    sep = c.float().cpu().numpy()[..., :C_out]
+    assert np.max(np.abs(sep - got) / (MATCH_REL * np.abs(ref_m) + 1e-3 * bound_m)) <= 2.0
+
+
+def test_fused_block_argument_errors_and_unsupported_shapes(cp):
+    for args in ((2, 64, 28, 28, 288, 64), (2, 256, 14, 14, 512, 64), (2, 64, 14, 14, 288, 320)):   # image too large, C_in, C_out
+        with pytest.raises(cp.CpruneError) as e:
+            cp.cprune_block_plan(*args)
+        assert e.value.status == 2
+    with pytest.raises(cp.CpruneError) as e:
+        cp.cprune_block_plan(2, 64, 14, 14, 288, 96, residual=True)        # a residual needs C_in == C_out
+    assert e.value.status == 1
+    a = cp.cprune_block_plan(2, 64, 14, 14, 288, 64, residual=True)
+    b = cp.cprune_block_plan(2, 64, 14, 14, 288, 64, residual=True)
+    assert a.handle.value == b.handle.value and a.unfused_bytes > 2 * a.algorithmic_bytes
+
+
+def test_mobilenet_v2_with_and_without_fused_blocks(cp):
+    from paper_2207_01260_b200.pipeline import PrunedNetwork
+    table = wl.mobilenet_v2()
+    weights = wl.model_weights(table)
+    x = wl.model_input(table, 4)
+    fused = PrunedNetwork(table, weights, 4, fuse_blocks=True)
+    plain = PrunedNetwork(table, weights, 4, fuse_blocks=False)
+    # the stride-1 blocks of the 14x14 and 7x7 stages, except the last one (320 filters do not fit one image's accumulator)
+    assert sorted(fused.blocks) == sorted(["b8_exp", "b9_exp", "b10_exp", "b11_exp", "b12_exp", "b13_exp", "b15_exp", "b16_exp"])
+    assert not PrunedNetwork(table, weights, 64).blocks and PrunedNetwork(table, weights, 2).blocks      # the default follows the batch
+    assert fused.model.launches == plain.model.launches - sum(3 - (2 if b.splits > 1 else 1) for b in fused.blocks.values())
+    a = fused.run(_dev(x)).cpu().numpy()
+    b = plain.run(_dev(x)).cpu().numpy()
+    cp.cprune_poll_device_status()
+    assert np.linalg.norm(a - b) <= 3e-3 * np.linalg.norm(b)
+    pw, _ = oracle.prune_model(table, weights)
+    ref = oracle.model_ref(table, pw, x, matched=True)
+    assert np.linalg.norm(a - ref) <= 1e-2 * np.linalg.norm(ref)
+    print("\nfused blocks: %s; launches %d -> %d" % (sorted(fused.blocks), plain.model.launches, fused.model.launches))
+
+
 def test_shared_selection_and_shortcut_pruned_resnet(cp):
     # dependency-aware pruning: one ranking for the layers whose outputs meet in a residual add
     ws = [wl.normal_f32(51, 1, (96, 20, 3, 3), 0.1), wl.normal_f32(51, 2, (96, 64, 1, 1), 0.1), wl.normal_f32(51, 3, (96, 7, 3, 3), 0.1)]
