@@ -140,6 +140,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="images per step and GPU (0: the workload's own batch; 1 gives the latency point)")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every launch from the host instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the 1.2 s sustained run (for profiler launch lists)")
     ap.add_argument("--no-task-times", action="store_true",
                     help="skip the per-task timing passes (and with them the roofline object); for profiler launch lists")
     ap.add_argument("--task", default=None,
@@ -255,7 +256,7 @@ def main():
 
     # ---------------- sustained: at least 1.2 s of back-to-back replays, so that the clock record covers the timed
     # kernels (the 20 to 50 steps above last a few milliseconds, far less than the 100 ms sampling period)
-    n_sus = max(args.steps, int(1.2 / max(ms / args.steps * 1e-3, 1e-6)) + 1)
+    n_sus = args.steps if args.no_sustained else max(args.steps, int(1.2 / max(ms / args.steps * 1e-3, 1e-6)) + 1)
     barrier()
     sus_sampler = ClockSampler(local_rank)
     sus_sampler.start()

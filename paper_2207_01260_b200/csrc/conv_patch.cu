@@ -959,6 +959,8 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
                 if (wstages > 8) wstages = 8;
             }
             if (dense && staging_bufs != 2) continue;
+            // the fused 3x3 pool runs on its own warps only beside two staging buffers, which is worth more than a deeper ring
+            if (pool3 && staging_bufs != 2 && pstages > 2) continue;
             const long long tiles = (long long)g.vN * tiles_per_img * tiles_n;
             const double waves = (double)((tiles + 147) / 148);
             double tile = tile_cycles(MT, FT, RS, cblks, ksteps_last, RB, Wp, TH, g.kR, resident != 0, acc_bufs);
