@@ -68,29 +68,35 @@ __device__ __forceinline__ float apply_act(float v, int act) {
     return v;
 }
 
-// 8 bf16 values carried in one 16-byte vector
+// 8 bf16 values carried in one 16-byte vector.  The members are plain words so that a copy of the struct is ONE 16-byte
+// load or store (with __nv_bfloat162 members, whose assignment is user-defined, it is four 4-byte ones).
 struct alignas(16) bf16x8 {
-    __nv_bfloat162 v[4];
+    uint32_t w[4];
 };
 
 __device__ __forceinline__ bf16x8 ldg8(const bf16x8 *p) {
     uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
-    return *reinterpret_cast<bf16x8 *>(&u);
+    bf16x8 r;
+    r.w[0] = u.x; r.w[1] = u.y; r.w[2] = u.z; r.w[3] = u.w;
+    return r;
 }
 
 __device__ __forceinline__ void unpack8(const bf16x8 &a, float *f) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        float2 t = __bfloat1622float2(a.v[i]);
-        f[2 * i] = t.x;
-        f[2 * i + 1] = t.y;
+        // a bf16 is the upper half of the float32 with the same value
+        f[2 * i] = __uint_as_float(a.w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(a.w[i] & 0xffff0000u);
     }
 }
 
 __device__ __forceinline__ bf16x8 pack8(const float *f) {
     bf16x8 r;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) r.v[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 t = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+        r.w[i] = *reinterpret_cast<const uint32_t *>(&t);
+    }
     return r;
 }
 

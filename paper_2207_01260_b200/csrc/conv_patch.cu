@@ -17,11 +17,15 @@
 // j >= Q are the S - 1 wrap-around columns: they are computed and thrown away.  A tile has MT
 // blocks of 128 slots (MT = 1 or 2, one accumulator each, both fed by the same filter stage).
 //
-//   warp 0       patch loads (one per channel block);
+//   warp 0       patch loads (one per channel block); with a residual, one more load per group of
+//                64 filters brings the residual tile in through the same ring;
 //   warps 1, 2   filter loads, one per (channel block, tap), taken in turn; small filter sets
 //                stay resident in shared memory for the whole kernel;
-//   warps 3, 12  tcgen05.mma issue, one warp per accumulator block;
-//   warps 4..11  epilogue: tcgen05.ld, bias (+ residual), activation, bf16 into a swizzled staging
+//   warps 3, 12  tcgen05.mma issue, one warp per accumulator block; the residual tile is added by
+//                one more MMA against a 64 x 64 identity held in shared memory (bf16 x 1.0 into an
+//                fp32 accumulator is exact), so the epilogue never touches global memory for it
+//                (the 1x1 instantiation, whose tile is flat, still adds it in the epilogue);
+//   warps 4..11  epilogue: tcgen05.ld, bias, activation, bf16 into a swizzled staging
 //                buffer, then ONE TMA store per group of 64 filters whose box is the tile's rows x
 //                Wp pixels (wrap-around columns, rows below the image and filters beyond k_pad lie
 //                outside the tensor map and are not written).  With a fused max-pool the staged
@@ -41,7 +45,7 @@ namespace cprune {
 
 constexpr int PK_THREADS = 13 * 32;       // general kernel: 5 role warps + 8 epilogue warps
 constexpr int PK_THREADS_DENSE = 21 * 32; // dense-staging kernel: 16 epilogue warps (its epilogue bounds the tile; it needs few registers)
-constexpr int PK_POOL_WARPS = 4;          // 3x3-pool kernel: these warps pool the staged tile while the epilogue warps stage the next one
+constexpr int PK_POOL_WARPS = 8;          // 3x3-pool kernel: these warps pool the staged tile while the epilogue warps stage the next one
 constexpr int PK_THREADS_POOL3 = (13 + PK_POOL_WARPS) * 32;
 // kernel instantiations
 constexpr int PK_GENERAL = 0, PK_DENSE = 1, PK_POOL3 = 2;
@@ -1012,12 +1016,12 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
 // 16-channel bf16 pixels, one per sf x sf block of input pixels, in rows of WP pixels of which the first pad_lo (and
 // whatever follows the image) are zero:
 //   out[n][h2][pad_lo + w2][(dy * sf + dx) * C + c] = x[n][sf * h2 + dy][sf * w2 + dx][c], other channels zero.
-// Eight threads per output pixel, two channels each: the 32 bytes of a pixel are written by neighbouring lanes.
+// Two threads per output pixel, eight channels (one 16-byte store) each.
 constexpr int RG_ROWS = 4;     // regrouped rows per block
 
 template <typename T>
 __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, int H, int W, int C, int c_mem, int sf, int pad_lo, int WP,
-                                                      __nv_bfloat162 *__restrict__ out) {
+                                                      uint4 *__restrict__ out) {
     pdl_trigger();
     pdl_wait();
     // one block per RG_ROWS regrouped rows of one image: their sf * RG_ROWS input rows are contiguous in memory and are
@@ -1042,26 +1046,40 @@ __global__ void __launch_bounds__(256) regroup_kernel(const T *__restrict__ x, i
     if (((reinterpret_cast<uintptr_t>(rows) | n_bytes) & 15) == 0) {
         const uint4 *src = reinterpret_cast<const uint4 *>(rows);
         uint4 *dst = reinterpret_cast<uint4 *>(rg_smem);
-        for (int i = threadIdx.x; i < (int)(n_bytes >> 4); i += blockDim.x) dst[i] = __ldg(src + i);
+        const int n16 = (int)(n_bytes >> 4);
+        // four loads in flight per thread: the block's latency is one round trip to memory, not one per 4 KB
+        for (int i0 = threadIdx.x; i0 < n16; i0 += 4 * 256) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * 256 < n16) v[u] = __ldg(src + i0 + u * 256);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i0 + u * 256 < n16) dst[i0 + u * 256] = v[u];
+        }
     } else {
         for (int i = threadIdx.x; i < n_elems; i += blockDim.x) srow[i] = rows[i];
     }
     __syncthreads();
-    __nv_bfloat162 *orow = out + ((size_t)n * H2 + h2_0) * WP * 8;
-    const int per_row = WP * 8;
+    uint4 *orow = out + ((size_t)n * H2 + h2_0) * WP * 2;
+    const int per_row = WP * 2;
     const int step = sf * c_mem;                         // input elements between neighbouring regrouped pixels
-    for (int r = 0; r < nrows; ++r) {
-        const T *in = srow + (size_t)r * row_elems;
-        for (int e = threadIdx.x; e < per_row; e += blockDim.x) {
-            const int pair = e & 7, w2 = (e >> 3) - pad_lo;
-            float v0 = 0.f, v1 = 0.f;
-            if (w2 >= 0 && w2 < W2) {
-                const int o0 = src_off[2 * pair], o1 = src_off[2 * pair + 1];
-                if (o0 >= 0) v0 = (float)in[o0 + w2 * step];
-                if (o1 >= 0) v1 = (float)in[o1 + w2 * step];
+    for (int e = threadIdx.x; e < nrows * per_row; e += blockDim.x) {
+        const int r = e / per_row, c = e - r * per_row;
+        const int half = c & 1, w2 = (c >> 1) - pad_lo;
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = 0.f;
+        if (w2 >= 0 && w2 < W2) {
+            const T *in = srow + (size_t)r * row_elems + w2 * step;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int o = src_off[half * 8 + k];
+                if (o >= 0) v[k] = (float)in[o];
             }
-            orow[(size_t)r * per_row + e] = __floats2bfloat162_rn(v0, v1);
         }
+        const bf16x8 q = pack8(v);
+        orow[e] = *reinterpret_cast<const uint4 *>(&q);
     }
 }
 
@@ -1116,10 +1134,10 @@ cprune_status regroup_stem_input(const cprune_plan *plan, const void *x, int x_i
     if (row_bytes > 48 * 1024) return CPRUNE_ERR_UNSUPPORTED;     // planning keeps such images off this path
     if (x_is_f32)
         CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<float>, dim3(blocks), dim3(256), row_bytes, st, (const float *)x, i.H, i.W, i.C, i.C, g.sf, g.pad_lo,
-                                         g.WP, (__nv_bfloat162 *)scratch));
+                                         g.WP, (uint4 *)scratch));
     else
         CPRUNE_CUDA_CHECK(launch_chained(regroup_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), row_bytes, st, (const __nv_bfloat16 *)x, i.H, i.W, i.C,
-                                         i.c_pad, g.sf, g.pad_lo, g.WP, (__nv_bfloat162 *)scratch));
+                                         i.c_pad, g.sf, g.pad_lo, g.WP, (uint4 *)scratch));
     return CPRUNE_OK;
 }
 
