@@ -31,6 +31,21 @@ struct DwParams {
 
 __device__ __forceinline__ uint32_t dw_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// a0 += x.lo * w.lo, a1 += x.hi * w.hi for two packed bf16 pairs: the mixed-precision fused multiply-add takes bf16
+// factors and a float32 addend.  A product of two bf16 values is exact in float32, so the result is the one
+// fmaf(float(x), float(w), a) gives, without the two conversions per pair.
+__device__ __forceinline__ void fma_bf16x2(float &a0, float &a1, uint32_t x, uint32_t w) {
+    asm("{\n\t"
+        ".reg .b16 xl, xh, wl, wh;\n\t"
+        "mov.b32 {xl, xh}, %2;\n\t"
+        "mov.b32 {wl, wh}, %3;\n\t"
+        "fma.rn.f32.bf16 %0, xl, wl, %0;\n\t"
+        "fma.rn.f32.bf16 %1, xh, wh, %1;\n\t"
+        "}"
+        : "+f"(a0), "+f"(a1)
+        : "r"(x), "r"(w));
+}
+
 template <int STRIDE>
 __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant__ CUtensorMap tm_x, const DwParams p) {
     extern __shared__ __align__(128) uint8_t dw_smem[];
@@ -68,12 +83,12 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
     const int cgg = cb * G + cg;             // channel group within the tensor
     const bool active = qq < p.TW && q0 + qq < p.Q && cgg < p.c8;
 
-    // filter taps (float32) and bias of this thread's 8 channels (overlaps the load)
-    float wf[9][8];
+    // filter taps (bf16 pairs, as packed) and bias of this thread's 8 channels (overlaps the load)
+    bf16x8 wq[9];
     float bf[8];
     if (active) {
 #pragma unroll
-        for (int t = 0; t < 9; ++t) unpack8(ldg8(p.w + (size_t)t * p.c8 + cgg), wf[t]);
+        for (int t = 0; t < 9; ++t) wq[t] = ldg8(p.w + (size_t)t * p.c8 + cgg);
 #pragma unroll
         for (int i = 0; i < 8; ++i) bf[i] = __ldg(p.b + cgg * 8 + i);
     }
@@ -123,8 +138,13 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
     };
 
     if (STRIDE == 1) {
-        // walk down the input rows; each row feeds the three output rows it overlaps
+        // walk down the input rows; each row feeds the three output rows it overlaps.  An input value is used three
+        // times here, so it is converted to float32 once (measured: faster than the mixed-precision form below, and
+        // than packed float32 pairs with rotating accumulators)
         const int rows = min(p.TH, p.P - p0);       // output rows of this tile
+        float wf[9][8];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) unpack8(wq[t], wf[t]);
         float a0[8], a1[8], a2[8];                  // accumulators of output rows h-2, h-1, h
 #pragma unroll
         for (int i = 0; i < 8; ++i) { a0[i] = bf[i]; a1[i] = bf[i]; a2[i] = bf[i]; }
@@ -146,6 +166,7 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
             for (int i = 0; i < 8; ++i) { a0[i] = a1[i]; a1[i] = a2[i]; a2[i] = bf[i]; }
         }
     } else {
+        // an input value is used once per output row here: the mixed-precision FMA saves its conversion
         for (int pp = 0; pp < p.TH && p0 + pp < p.P; ++pp) {
             float acc[8];
 #pragma unroll
@@ -155,10 +176,9 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const __grid_constant
                 const bf16x8 *row = patch + ((size_t)(pp * STRIDE + r) * p.IW + qq * STRIDE) * G;
 #pragma unroll
                 for (int s = 0; s < 3; ++s) {
-                    float xf[8];
-                    unpack8(row[s * G], xf);
+                    const bf16x8 x = row[s * G];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(xf[i], wf[r * 3 + s][i], acc[i]);
+                    for (int j = 0; j < 4; ++j) fma_bf16x2(acc[2 * j], acc[2 * j + 1], x.w[j], wq[r * 3 + s].w[j]);
                 }
             }
             finish(acc, pp);
