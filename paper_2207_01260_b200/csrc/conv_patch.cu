@@ -72,6 +72,7 @@ struct PatchParams {
     int w_stage_bytes;     // shared memory of one filter stage (FT rows, rounded up to 1024 bytes)
     int rb16;              // bytes per pixel row in shared memory / 16: 8 (64 channels) or 2 (16 channels, regrouped stems)
     int dense;             // the staged tile is [slot][k_pad] as in memory and leaves by one bulk copy (flat tasks, one filter tile)
+    int dense_pitch;       // ... bytes per slot in the staging buffer: k_pad * 2, or 16 more (then the tile leaves by a tiled copy)
     int stage_bytes;       // shared memory of one staging buffer
     int res_blocks;        // residual added on the tensor core: 64-filter blocks of the residual tile per item (0: none)
     const float *bias;
@@ -529,12 +530,19 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // the epilogue has nothing to do with it.  Dense staging: the residual of tile item_ (tiles_n == 1, one row of
         // tiles) is one contiguous range of memory, arrives in the staging buffer the tile will use and is added in place.
         const bool with_res = DENSE && p.res != nullptr;
+        const bool dense_tiled = DENSE && p.dense_pitch != p.k_pad * 2;
         auto load_residual_dense = [&](int item_, uint32_t counter) {
             const int q0_ = item_ * p.step_w;
             const uint32_t bytes = (uint32_t)min(p.TW, p.Q - q0_) * (uint32_t)p.k_pad * 2u;
             const uint32_t b = counter & 1u;
-            mbar_expect_tx(res_full(b), bytes);
-            bulk_load(staging0 + b * stage_buf_bytes, p.res + (size_t)q0_ * p.k_pad, bytes, res_full(b));
+            if (dense_tiled) {
+                // the box is the whole tile, one piece wider than the tensor: what lies outside arrives as zeros
+                mbar_expect_tx(res_full(b), (uint32_t)p.TW * (uint32_t)p.dense_pitch);
+                tma_load_4d(staging0 + b * stage_buf_bytes, &tm_res, res_full(b), 0, q0_, 0, 0);
+            } else {
+                mbar_expect_tx(res_full(b), bytes);
+                bulk_load(staging0 + b * stage_buf_bytes, p.res + (size_t)q0_ * p.k_pad, bytes, res_full(b));
+            }
         };
         if (with_res && store_thread && (int)blockIdx.x < total_items) {
             pdl_wait();        // the residual is the result of an earlier kernel of the chain
@@ -555,11 +563,13 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.MT * p.FT);
             if constexpr (DENSE) {
                 // Flat task with one filter tile: the tile's output is ONE contiguous range of y (slot-major, k_pad filters
-                // per slot).  It is staged in exactly that layout and leaves by a single bulk copy; a residual arrives the
-                // same way.  (Rows of k_pad * 2 bytes: the 16-byte pieces of eight neighbouring slots fall in distinct banks.)
+                // per slot).  With an odd number of 16-byte pieces per slot it is staged in exactly that layout (the pieces
+                // of eight neighbouring slots fall in distinct banks) and leaves by a single bulk copy; a residual arrives
+                // the same way.  With an even number the staged slots are one piece longer, and the tile moves by a tiled
+                // copy whose box is that one piece wider than the tensor: the piece outside is not written (read as zeros).
                 const uint32_t b = group_counter & 1u;
                 uint8_t *buf = smem + (staging0 - base) + b * stage_buf_bytes;
-                const uint32_t pitch = (uint32_t)p.k_pad * 2u;
+                const uint32_t pitch = (uint32_t)p.dense_pitch;
                 if (with_res) {
                     ok = __all_sync(0xffffffffu, mbar_wait(res_full(b), (group_counter >> 1) & 1u, abort_flag, p.status, false));
                     if (!ok) break;
@@ -612,7 +622,8 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (!ok) break;
                 if (store_thread) {
                     const int rows = min(p.TW, p.Q - q0);
-                    bulk_store(p.y + (size_t)q0 * p.k_pad, staging0 + b * stage_buf_bytes, (uint32_t)rows * pitch);
+                    if (dense_tiled) tma_store_4d(&tm_y, staging0 + b * stage_buf_bytes, 0, q0, 0, 0);
+                    else bulk_store(p.y + (size_t)q0 * p.k_pad, staging0 + b * stage_buf_bytes, (uint32_t)rows * pitch);
                     tma_store_commit();
                     if (with_res && item + (int)gridDim.x < total_items) load_residual_dense(item + gridDim.x, group_counter + 1);
                 }
@@ -932,8 +943,10 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             // won on every ResNet-18 shape (26.5 vs 27.8 us, 21.1 vs 22.5 us, 21.9 vs 21.7 us).
             const int res_blocks_plan = plan->opts.residual ? (FT + 63) / 64 : 0;
           for (int pstages = ps_max; pstages >= 2; --pstages) {
-            const int dense_bytes = round_up(128 * MT * i.k_pad * 2, 1024);
-            const int dense = g.flat && tiles_n == 1 && (((i.k_pad >> 3) & 1) || i.k_pad == 16) && dense_bytes <= 40 * 1024;
+            const int dense_pitch = ((((i.k_pad >> 3) & 1) || i.k_pad == 16) ? i.k_pad : i.k_pad + 8) * 2;
+            const int dense_bytes = round_up(128 * MT * dense_pitch, 1024);
+            const int dense = g.flat && tiles_n == 1 && dense_pitch <= 512 && dense_bytes <= 48 * 1024 &&
+                              (dense_pitch == i.k_pad * 2 || !plan->opts.residual);
             // a residual is added on the tensor core (identity operand in shared memory), except with dense staging,
             // where it arrives in the staging buffer
             const int ident_bytes = (plan->opts.residual && !dense) ? PK_IDENT_BYTES : 0;
@@ -941,8 +954,8 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             const int budget = 227 * 1024 - fixed;
             const int sb_max = 2, sb_min = 1;
             const int w_stage = round_up(FT * RB, 1024);
-            // flat tasks with one filter tile stage the tile as it lies in memory (k_pad filters per pixel) when that fits
-            // and the pixel pitch is an odd number of 16-byte pieces (no bank conflicts between neighbouring pixels;
+            // flat tasks with one filter tile stage the tile as it lies in memory (k_pad filters per pixel) when that fits,
+            // with the pixel pitch made an odd number of 16-byte pieces (no bank conflicts between neighbouring pixels;
             // 32-byte pixels conflict two-way and still gain, measured)
             const int stage_bytes = dense ? dense_bytes : MT * PK_BLOCK_BYTES;
             int staging_bufs = sb_max, wstages = 0, resident = 0;
@@ -973,7 +986,7 @@ cprune_status plan_conv_patch(cprune_plan *plan) {
             if (resident) t += RS * cblks * FT;    // one-time filter load
             if (t < best) {
                 best = t;
-                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org, pstages, dense, stage_bytes};
+                bt = {MT, TH, FT, tiles_n, tiles_per_img, wstages, resident, acc_bufs, staging_bufs, patch_bytes, TW, tiles_w, step_h, step_w, org, pstages, dense, stage_bytes, dense_pitch};
             }
             break;      // the deepest ring that fits
           }
@@ -1197,8 +1210,10 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
                                                 (unsigned long long)g.vN};
             const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)g.vOW * i.k_pad * 2,
                                                    (unsigned long long)g.vOH * g.vOW * i.k_pad * 2};
-            const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
-            cprune_status s = encode_tiled_bf16_swz(&plan->tm_y, y, 4, dims, strides, box, 128, false);
+            const bool dense_tiled = t.dense && t.dense_pitch != i.k_pad * 2;      // the whole staged tile, unswizzled
+            const unsigned box[4] = {dense_tiled ? (unsigned)(t.dense_pitch / 2) : 64u, dense_tiled ? (unsigned)t.TW : (unsigned)Wp,
+                                     dense_tiled ? 1u : (unsigned)t.TH, 1};
+            cprune_status s = encode_tiled_bf16_swz(&plan->tm_y, y, 4, dims, strides, box, dense_tiled ? 0 : 128, false);
             if (s != CPRUNE_OK) return s;
             plan->map_y = y;
         }
@@ -1207,8 +1222,10 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
                                                 (unsigned long long)g.vN};
             const unsigned long long strides[3] = {(unsigned long long)i.k_pad * 2, (unsigned long long)g.vQ * i.k_pad * 2,
                                                    (unsigned long long)g.vP * g.vQ * i.k_pad * 2};
-            const unsigned box[4] = {64, (unsigned)Wp, (unsigned)t.TH, 1};
-            cprune_status s = encode_tiled_bf16_swz(&plan->tm_res, res, 4, dims, strides, box, 128, true);
+            const bool dense_tiled = t.dense && t.dense_pitch != i.k_pad * 2;
+            const unsigned box[4] = {dense_tiled ? (unsigned)(t.dense_pitch / 2) : 64u, dense_tiled ? (unsigned)t.TW : (unsigned)Wp,
+                                     dense_tiled ? 1u : (unsigned)t.TH, 1};
+            cprune_status s = encode_tiled_bf16_swz(&plan->tm_res, res, 4, dims, strides, box, dense_tiled ? 0 : 128, true);
             if (s != CPRUNE_OK) return s;
             plan->map_res = res;
         }
@@ -1246,7 +1263,7 @@ cprune_status launch_conv_patch(cprune_plan *plan, const void *x, const void *w,
     p.patch_bytes = t.patch_bytes;
     p.patch_box_bytes = Wp * (t.TH + g.kR - 1) * 128;
     p.rb16 = 8;
-    p.dense = t.dense; p.stage_bytes = t.stage_bytes;
+    p.dense = t.dense; p.stage_bytes = t.stage_bytes; p.dense_pitch = t.dense_pitch;
     p.w_stage_bytes = t.FT * 128;
     p.bias = b;
     // dense staging takes the residual through the staging buffer; everywhere else the MMA warps add it

@@ -17,6 +17,7 @@ struct PatchTiling {
     int pstages;                            // depth of the patch ring
     int dense;                              // flat tasks: a tile's output is staged as it lies in memory and stored by one bulk copy
     int stage_bytes;                        // shared memory of one staging buffer
+    int dense_pitch;                        // dense staging: bytes between neighbouring pixels in the staging buffer
 };
 
 struct cprune_plan {

@@ -219,7 +219,7 @@ const char *cprune_status_string(cprune_status s) {
 
 const char *cprune_last_cuda_error(void) { return t_last_error.c_str(); }
 
-int cprune_padded_channels(int C) { return C <= 0 ? 0 : (C + 7) / 8 * 8; }
+int cprune_padded_channels(int C) { return C <= 0 ? 0 : (C <= 128 ? (C + 7) / 8 * 8 : (C + 15) / 16 * 16); }
 
 size_t cprune_select_workspace_bytes(int K) {
     if (K <= 0) return 0;

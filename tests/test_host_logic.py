@@ -32,7 +32,7 @@ def test_status_strings_and_padding(cp):
     L = cp.lib()
     assert L.cprune_status_string(0) == b"ok"
     assert len({L.cprune_status_string(i) for i in range(8)}) == 8
-    assert [cp.cprune_padded_channels(c) for c in (1, 3, 8, 9, 44, 45, 243, 358)] == [8, 8, 8, 16, 48, 48, 248, 360]
+    assert [cp.cprune_padded_channels(c) for c in (1, 3, 8, 9, 44, 45, 72, 128, 129, 243, 358)] == [8, 8, 8, 16, 48, 48, 72, 128, 144, 256, 368]
     assert cp.cprune_select_workspace_bytes(0) == 0 and cp.cprune_select_workspace_bytes(1280) >= 1280 * 12
 
 
@@ -69,9 +69,9 @@ def test_plan_shapes_and_families(cp):
     # a pointwise stride-1 task with many pixels is planned as a flat matrix product: tiles of 128 or 256 pixels
     f = cp.cprune_task_plan(64, 24, 56, 56, 108, 1, 1, 1, 0, activation="relu6")
     assert f.variant == 1 and f.tile_m in (128, 256) and f.tiles_m == -(-64 * 56 * 56 // f.tile_m) and f.workspace_bytes == 0
-    # one filter tile and a pixel pitch of an odd number of 16-byte pieces (or 32 bytes): the tile is staged as it lies in
-    # memory (variant 2); a pitch that would conflict in shared memory, or several filter tiles, keep the tiled stores
-    for K, want in ((72, 2), (24, 2), (16, 2), (40, 2), (32, 1), (64, 1), (108, 1), (300, 1)):
+    # one filter tile: the tile is staged pixel by pixel as it lies in memory (variant 2; the staged pixels are made an odd
+    # number of 16-byte pieces long); a tile too large to stage that way, or several filter tiles, keep the tiled stores
+    for K, want in ((72, 2), (24, 2), (16, 2), (40, 2), (32, 2), (64, 2), (108, 1), (300, 1)):
         d = cp.cprune_task_plan(64, 48, 56, 56, K, 1, 1, 1, 0, activation="relu6")
         assert d.variant == want, (K, d.variant)
     # the ResNet stem with its 3x3 stride-2 pool: pooled output extent, pool fused (no unpooled copy in the workspace,
