@@ -30,7 +30,7 @@ import numpy as np  # noqa: E402
 
 # DRAM bytes (read + write) of all launches of a kernel in one model pass, from the ncu captures summarised under profiles/
 # (conv_patch_resnet18_b64_dram_traffic.md); absent where no capture of the current kernel exists.
-DRAM_BYTES_PER_STEP = {("resnet18", "conv_patch_kernel"): 258.4e6}
+DRAM_BYTES_PER_STEP = {("resnet18", "conv_patch_kernel"): 258.9e6}
 
 WORKLOADS = {"resnet18": ("resnet18", 64), "mobilenet_v2": ("mobilenet_v2", 64), "vgg16_cifar": ("vgg16_cifar", 128)}
 
