@@ -166,8 +166,9 @@ typedef struct {
                                  lies in memory and stored by a single bulk copy */
     int splits;               /* slices of the reduction that go to different CTAs (1: no split); > 1 adds a second launch */
     /* How the program splits the two iterators that run over the filters (paper Sec. 3.5): the compute iterator
-     * (filter tiles x instruction-sized groups per tile) and the store iterator (filter tiles x 16-byte pieces per
-     * tile); each count stands for `unit` filters that one instruction or one store handles and that cannot shrink. */
+     * (filter tiles x instruction-sized groups per tile) and the store iterator (filter tiles x pieces of the memory
+     * layout's channel granule per tile: 8 filters up to 128 filters, 16 above, see cprune_padded_channels); each
+     * count stands for `unit` filters that one instruction or one store handles and that cannot shrink. */
     int split_compute[2], unit_compute;
     int split_store[2], unit_store;
     double est_us;            /* the planner's own estimate of the task's time (its cost model, microseconds) */

@@ -83,11 +83,12 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
     i.splits = family == CPRUNE_KERNEL_TENSOR ? pl->splits : 1;
     if (family == CPRUNE_KERNEL_TENSOR && (pl->patch || pl->orient == 0)) {
         // filters on the MMA's column side: tiles_n tiles of tile_n filters, built from 16-filter instruction groups
-        // (64-filter groups when there are several tiles: tiles end on store-box boundaries), stored in 16-byte pieces
+        // (64-filter groups when there are several tiles: tiles end on store-box boundaries), stored in pieces of the
+        // memory layout's granule (8 filters = 16 bytes up to 128 filters, 16 filters above)
         i.unit_compute = i.tiles_n > 1 ? 64 : 16;
         i.split_compute[0] = i.tiles_n; i.split_compute[1] = i.tile_n / i.unit_compute;
-        i.unit_store = 8;
-        i.split_store[0] = i.tiles_n; i.split_store[1] = i.tile_n / 8;
+        i.unit_store = i.K > 128 ? 16 : 8;
+        i.split_store[0] = i.tiles_n; i.split_store[1] = i.tile_n / i.unit_store;
     } else if (family == CPRUNE_KERNEL_DEPTHWISE) {
         // channel blocks (CTAs along the channels) x channel groups of 8 per CTA
         const int c8 = i.c_pad / 8;
@@ -98,10 +99,10 @@ static cprune_status build_plan(const PlanKey &key, cprune_plan **out) {
         pl->est_us = i.algorithmic_bytes / 3.0e6 + 4.0;
     } else {
         // filters on the 128-row side of the MMA (any count up to 128 costs the same) or one thread per 8 filters:
-        // the filter axis is only cut into the 8-filter pieces of the memory layout
-        i.unit_compute = i.unit_store = 8;
+        // the filter axis is only cut into the pieces of the memory layout (8 filters up to 128 filters, 16 above)
+        i.unit_compute = i.unit_store = i.K > 128 ? 16 : 8;
         i.split_compute[0] = i.split_store[0] = 1;
-        i.split_compute[1] = i.split_store[1] = i.k_pad / 8;
+        i.split_compute[1] = i.split_store[1] = i.k_pad / i.unit_store;
         if (family == CPRUNE_KERNEL_DIRECT) pl->est_us = i.flops / 15.0e6 + 4.0;
     }
     i.variant = (family == CPRUNE_KERNEL_TENSOR && pl->patch) ? (pl->pt.dense ? 2 : 1) : 0;

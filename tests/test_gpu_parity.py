@@ -212,13 +212,16 @@ def test_pointwise_tasks_as_flat_matrix_products(cp):
     check_task(cp, 3, 108, 57, 59, 24, 1, 1, 0, act="none", with_res=True, kernel="tensor")
     check_task(cp, 5, 72, 40, 41, 300, 1, 1, 0, act="relu", kernel="tensor")
     check_task(cp, 64, 320, 7, 7, 1280, 1, 1, 0, act="relu6", kernel="tensor")
-    # one filter tile and a pixel pitch of an odd number of 16-byte pieces (or 32 bytes): the tile is staged as it lies
-    # in memory and leaves by one bulk copy (one and two 64-filter groups, with and without residual, ragged last tile)
-    for case in ((12, 16, 50, 53, 72, "relu6", False), (6, 32, 47, 50, 16, "none", False), (4, 150, 45, 46, 40, "relu6", True),
-                 (8, 48, 45, 46, 133, "relu", True)):
-        N, C, H, W, K, act, res = case
+    # one filter tile: the tile is staged pixel by pixel as it lies in memory (variant 2).  A pixel pitch of an odd number of
+    # 16-byte pieces (or 32 bytes) leaves by one bulk copy (one and two 64-filter groups, with and without residual, ragged
+    # last tile); an even number is staged one piece longer and leaves by one tiled copy whose box is wider than the tensor
+    # (without residual; with one such tasks keep the 64-filter-wide stores of variant 1)
+    for case in ((12, 16, 50, 53, 72, "relu6", False, 2), (6, 32, 47, 50, 16, "none", False, 2), (4, 150, 45, 46, 40, "relu6", True, 2),
+                 (8, 48, 45, 46, 88, "relu", True, 2), (8, 48, 45, 46, 133, "relu", False, 2), (5, 24, 44, 45, 64, "relu", False, 2),
+                 (7, 40, 33, 35, 32, "relu6", False, 2), (8, 48, 45, 46, 133, "relu", True, 1), (5, 24, 44, 45, 64, "none", True, 1)):
+        N, C, H, W, K, act, res, variant = case
         plan = check_task(cp, N, C, H, W, K, 1, 1, 0, act=act, with_res=res, kernel="tensor")
-        assert plan.variant == 2, case
+        assert plan.variant == variant, case
 
 
 def test_stems_on_the_patch_kernel(cp):
