@@ -896,8 +896,7 @@ cprune_status plan_conv_tensor(cprune_plan *plan) {
     return CPRUNE_OK;
 }
 
-static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w, void *y, const void *res,
-                                 cudaStream_t stream) {
+static cprune_status encode_maps(cprune_plan *plan, const void *x, const void *w, void *y, const void *res) {
     const cprune_plan_info &i = plan->info;
     cprune_status st = load_driver_entry_points();
     if (st != CPRUNE_OK) return st;
@@ -1014,7 +1013,7 @@ cprune_status launch_conv_tensor(cprune_plan *plan, const void *x, const void *w
     {
         std::lock_guard<std::mutex> lock(plan->mu);
         if (plan->map_x != x || plan->map_w != w || plan->map_y != y || (mma_res && plan->map_res != res)) {
-            cprune_status s = encode_maps(plan, x, w, y, res, st);
+            cprune_status s = encode_maps(plan, x, w, y, res);
             if (s != CPRUNE_OK) return s;
         }
         std::memcpy(&tm_x, &plan->tm_a, sizeof(CUtensorMap));
