@@ -402,7 +402,7 @@ conv_patch_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     } else if (SPLIT && warp > MMA_WARP2) {
         // ------------------------------------------------------------------ 3x3 stride-2 pooling of staged groups
         // The tile computed conv rows p0 .. p0 + TH - 1 (p0 odd or -1) and holds the windows of (TH - 1) / 2 x (TW - 1) / 2
-        // pooled pixels, all nine slots of each inside the staged tile.  A thread handles up to four (pooled pixel,
+        // pooled pixels, all nine slots of each inside the staged tile.  A thread handles up to 512 / (32 * PK_POOL_WARPS) (pooled pixel,
         // 8 filters) items, the same ones in every tile: the shared-memory offsets of their window slots are worked out once.
         const int ctid = threadIdx.x - (MMA_WARP2 + 1) * 32;
         constexpr int ITEMS = 512 / (PK_POOL_WARPS * 32);
